@@ -1,0 +1,131 @@
+"""Seeded synthetic inputs for one GSWA layer.
+
+This module only draws random tensors and rounds them to a storage type.  It
+holds none of the method's arithmetic, so both the CUDA path and the CPU
+checker can be fed from it without sharing anything else.
+
+Recipe (stands in for the paper's DIV2K training patches and test images,
+Sec. "Experimental Setup"): activations entering the attention layer follow a
+LayerNorm (Eq. 4), hence x ~ N(0,1); projection weights and the
+relative-position bias table ~ N(0, 0.02^2); projection biases zero unless a
+test asks otherwise; upstream gradient dy ~ N(0,1).  For bf16 workloads every
+sample is rounded to the nearest bf16 value (ties to even) before anybody sees
+it, and returned as float32 holding exactly that value.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, Tuple
+
+import numpy as np
+
+
+@dataclass(frozen=True)
+class LayerConfig:
+    """Shape of one GSWA layer call (notation of Sec. "Group Shifted Window Attention")."""
+
+    name: str
+    B: int
+    H: int
+    W: int
+    C: int
+    num_heads: int
+    window: int                      # M
+    group_heads: Tuple[int, ...]     # heads per group, consecutive
+    group_shift: Tuple[int, ...]     # cyclic shift of each group (0 = plain windows)
+    dtype: str = "bf16"              # "f32" | "bf16"
+    seed: int = 0
+    layers: int = 1                  # stacked-inference workloads call the layer this many times
+    backward: bool = True
+    bias_std: float = 0.0            # std of b_qkv / b_proj (0 in the paper-shaped workloads)
+
+    @property
+    def tokens(self) -> int:
+        return self.B * self.H * self.W
+
+    @property
+    def head_dim(self) -> int:
+        return self.C // self.num_heads
+
+
+# The workloads the layer is measured and checked on.  Batch 16..256 and C=60
+# are the paper's training batch sizes and lightweight width; 64x64 patches,
+# C=180 and window 8 are the classical-SR shape of the same model family.
+CONFIGS: Dict[str, LayerConfig] = {
+    "c1": LayerConfig("c1", 1, 16, 16, 60, 6, 8, (3, 3), (0, 4), dtype="f32", seed=0),
+    "c2": LayerConfig("c2", 64, 64, 64, 60, 6, 8, (3, 3), (0, 4), seed=2),
+    "c3": LayerConfig("c3", 32, 64, 64, 180, 6, 8, (3, 3), (0, 4), seed=3),
+    "cM": LayerConfig("cM", 64, 64, 64, 180, 6, 8, (3, 3), (0, 4), seed=6),
+    "c4": LayerConfig("c4", 256, 64, 64, 180, 6, 8, (3, 3), (0, 4), seed=4),
+    "c5": LayerConfig("c5", 1, 512, 512, 180, 6, 8, (3, 3), (0, 4), seed=5, layers=6, backward=False),
+}
+
+
+def round_to_bf16(a: np.ndarray) -> np.ndarray:
+    """Round float32 values to the nearest bf16 (ties to even); result stays float32."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    u = a.view(np.uint32)
+    bias = ((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF)
+    r = (u + bias) & np.uint32(0xFFFF0000)
+    return r.view(np.float32)
+
+
+def to_bf16_bits(a: np.ndarray) -> np.ndarray:
+    """Upper 16 bits of already-bf16-representable float32 values, as uint16."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return (a.view(np.uint32) >> np.uint32(16)).astype(np.uint16)
+
+
+def from_bf16_bits(b: np.ndarray) -> np.ndarray:
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+_TENSOR_STREAM = {"x": 1, "w_qkv": 2, "b_qkv": 3, "w_proj": 4, "b_proj": 5, "bias_table": 6, "dy": 7}
+
+
+def _normal(seed: int, layer: int, name: str, shape, std: float) -> np.ndarray:
+    ss = np.random.SeedSequence([int(seed), int(layer), _TENSOR_STREAM[name]])
+    rng = np.random.Generator(np.random.Philox(ss))
+    out = rng.standard_normal(size=shape, dtype=np.float32)
+    if std != 1.0:
+        out *= np.float32(std)
+    return out
+
+
+def make_inputs(cfg: LayerConfig, layer: int = 0, batch: int | None = None,
+                tensors=("x", "w_qkv", "b_qkv", "w_proj", "b_proj", "bias_table", "dy")) -> Dict[str, np.ndarray]:
+    """Draw the tensors of one layer call as float32 arrays.
+
+    `batch` overrides cfg.B with a smaller leading count (the first `batch`
+    images of the full draw are NOT reproduced; it is a separate, equally
+    distributed draw) -- used for bounded CPU samples.
+    """
+    B = cfg.B if batch is None else int(batch)
+    C, M, nh = cfg.C, cfg.window, cfg.num_heads
+    shapes = {
+        "x": ((B, cfg.H, cfg.W, C), 1.0),
+        "w_qkv": ((3 * C, C), 0.02),
+        "b_qkv": ((3 * C,), cfg.bias_std),
+        "w_proj": ((C, C), 0.02),
+        "b_proj": ((C,), cfg.bias_std),
+        "bias_table": (((2 * M - 1) ** 2, nh), 0.02),
+        "dy": ((B, cfg.H, cfg.W, C), 1.0),
+    }
+    out = {}
+    for name in tensors:
+        shape, std = shapes[name]
+        if std == 0.0:
+            a = np.zeros(shape, dtype=np.float32)
+        else:
+            a = _normal(cfg.seed, layer, name, shape, std)
+        if cfg.dtype == "bf16":
+            a = round_to_bf16(a)
+        out[name] = a
+    return out
+
+
+def layer_groups(cfg: LayerConfig, layer: int) -> Tuple[Tuple[int, ...], Tuple[int, ...]]:
+    """Head-group split of the `layer`-th stacked layer: odd layers swap which group shifts."""
+    if layer % 2 == 0:
+        return cfg.group_heads, cfg.group_shift
+    return cfg.group_heads, tuple(reversed(cfg.group_shift))
