@@ -1,0 +1,132 @@
+/*
+ * libgswa: Group Shifted Window Attention (GSWA) for NVIDIA B200 (sm_100a).
+ *
+ * One attention layer of AgileIR (arXiv 2409.06206), Sec. "Group Shifted Window
+ * Attention": the heads of a window-attention layer are split into groups; a
+ * group with shift 0 attends inside plain non-overlapping M x M windows
+ * (GW-MSA), a group with shift s > 0 attends after a cyclic shift of the
+ * feature map under the shifted-window mask (GSW-MSA); every head adds a
+ * learnable relative-position bias (Sec. "Learnable Relative Shifted Bias");
+ * the heads are concatenated and projected (Eq. 6, Eq. 7).  Forward and the
+ * training backward are provided; the backward recomputes the attention
+ * weights per window and never stores an M^2 x M^2 matrix.
+ *
+ * Plain C ABI.  Unless a parameter says "host", every pointer is a DEVICE
+ * pointer owned by the caller, 16-byte aligned, valid until the work enqueued
+ * on `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream) has
+ * finished.  Except where stated the library allocates no device memory and
+ * keeps no state between calls.  Every function returns GSWA_OK (0) or a
+ * negative gswa_status; argument errors are reported before anything is
+ * enqueued; nothing throws, traps or asserts on the device.
+ *
+ * Tensor conventions (the paper leaves them open):
+ *   x, y, dy, dx      [B,H,W,C], C fastest.
+ *   w_qkv             [3C, C] row-major (out, in); rows ordered q | k | v, head-major inside each.
+ *   b_qkv             [3C] or NULL (= zeros).
+ *   w_proj, b_proj    [C, C] (out, in), [C] or NULL.
+ *   bias_table        [(2M-1)^2, num_heads]; row (a_p-a_q+M-1)(2M-1) + (c_p-c_q+M-1) for query slot
+ *                     (a_p,c_p) and key slot (a_q,c_q) of a window.
+ *   q k^T is scaled by head_dim^-1/2; softmax runs over keys; the mask removes pairs (weight exactly 0).
+ *   cyclic shift by s: shifted[i',j'] = x[(i'+s) mod H, (j'+s) mod W].
+ * All of x, y, dy, dx, weights, biases and the table have the element type
+ * `dtype`; parameter gradients are always float32.
+ */
+#ifndef GSWA_H_
+#define GSWA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum gswa_status {
+  GSWA_OK = 0,
+  GSWA_ERR_NULL = -1,        /* a required pointer is NULL                                  */
+  GSWA_ERR_SHAPE = -2,       /* inconsistent sizes (H or W not a multiple of M, bad groups) */
+  GSWA_ERR_ALIGN = -3,       /* a device pointer is not 16-byte aligned                     */
+  GSWA_ERR_UNSUPPORTED = -4, /* valid but not implemented (e.g. qk_dim != head_dim)         */
+  GSWA_ERR_WORKSPACE = -5,   /* scratch / saved buffer too small                            */
+  GSWA_ERR_CUDA = -6         /* a CUDA runtime call or launch failed                        */
+} gswa_status;
+
+enum { GSWA_F32 = 0, GSWA_BF16 = 1 };
+
+enum {
+  GSWA_FLAG_ACCUMULATE = 1u, /* add into the parameter gradients instead of overwriting them */
+  GSWA_FLAG_GENERIC = 2u     /* force the shape-generic CUDA-core kernels (no tensor-core fast path) */
+};
+
+/* Layer description (host memory, read during the call only). */
+typedef struct gswa_desc {
+  int32_t B, H, W, C;         /* x is [B,H,W,C]                                               */
+  int32_t num_heads;          /* C % num_heads == 0; head_dim = C / num_heads                 */
+  int32_t window;             /* M; H % M == 0 and W % M == 0                                 */
+  int32_t num_groups;         /* G >= 1                                                       */
+  const int32_t* group_heads; /* host [G]; consecutive heads per group; sums to num_heads     */
+  const int32_t* group_shift; /* host [G]; 0 <= s < M; 0 = plain windows, no mask             */
+  int32_t dtype;              /* GSWA_F32 or GSWA_BF16                                        */
+  int32_t qk_dim, v_dim;      /* per-head widths; 0 = head_dim. Other values: GSWA_ERR_UNSUPPORTED */
+  uint32_t flags;             /* GSWA_FLAG_*                                                  */
+} gswa_desc;
+
+/* Buffer sizes for a layer description.
+ *   saved_bytes          forward -> backward carry (projected q,k,v, attention output, row log-sum-exp).
+ *   fwd_scratch_bytes    scratch of gswa_forward when `saved` is given.
+ *   infer_scratch_bytes  scratch of gswa_forward when `saved` is NULL (the carry then lives in scratch).
+ *   bwd_scratch_bytes    scratch of gswa_backward.
+ * Any output pointer may be NULL. */
+int gswa_workspace_query(const gswa_desc* desc, size_t* saved_bytes, size_t* fwd_scratch_bytes,
+                         size_t* infer_scratch_bytes, size_t* bwd_scratch_bytes);
+
+/* Forward pass, Eq. 6 and Eq. 7 with the window mask and relative bias:
+ *   y = Concat_h[ softmax(q_h k_h^T / sqrt(d) + B_h + mask) v_h ] W^P + b^P,  (q|k|v) = x W_qkv^T + b_qkv.
+ * `saved` (saved_bytes) receives what gswa_backward needs, or is NULL for inference.
+ * Contents of `scratch` are undefined afterwards.  Asynchronous on `cuda_stream`. */
+int gswa_forward(const gswa_desc* desc, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
+                 const void* b_proj, const void* bias_table, void* y, void* saved, void* scratch,
+                 size_t scratch_bytes, void* cuda_stream);
+
+/* Backward pass (reverse mode of gswa_forward; the paper's stated target is the memory of
+ * back-propagation).  `saved` is the buffer written by gswa_forward for the same desc and inputs.
+ * Writes dx (element type `dtype`) and the float32 parameter gradients dw_qkv[3C,C], db_qkv[3C],
+ * dw_proj[C,C], db_proj[C], dbias_table[(2M-1)^2, num_heads]; each gradient pointer may be NULL to
+ * skip it (dx included).  Gradients are overwritten unless GSWA_FLAG_ACCUMULATE is set.  Float32
+ * reductions use atomics: results are reproducible to rounding, not bitwise. */
+int gswa_backward(const gswa_desc* desc, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
+                  const void* bias_table, const void* saved, const void* dy, void* dx, float* dw_qkv,
+                  float* db_qkv, float* dw_proj, float* db_proj, float* dbias_table, void* scratch,
+                  size_t scratch_bytes, void* cuda_stream);
+
+/* Index maps of group `group`, computed on the device by the same routines the kernels use
+ * (Sec. "Patch Embedding" window partition; cyclic shift and window mask of GSW-MSA).  All int32,
+ * any pointer may be NULL:
+ *   win[H*W], slot[H*W], region[H*W]   per ORIGINAL token (i,j): window number in the shifted frame,
+ *                                      slot inside it (row-major M x M), mask label 3*r(i')+r(j')
+ *                                      with r = 0 on [0,n-M), 1 on [n-M,n-s), 2 on [n-s,n);
+ *   token_of[H*W]                      inverse map: token_of[win*M*M + slot] = i*W + j;
+ *   rel_index[M^2 * M^2]               bias-table row for (query slot, key slot). */
+int gswa_index_maps(const gswa_desc* desc, int32_t group, int32_t* win, int32_t* slot, int32_t* region,
+                    int32_t* token_of, int32_t* rel_index, void* cuda_stream);
+
+/* One training step on HOST buffers: copies x, the parameters and dy to the device arena, runs
+ * gswa_forward + gswa_backward, copies y, dx and the parameter gradients back, and waits for the
+ * stream.  All tensor pointers are HOST pointers (pinned memory makes the copies asynchronous);
+ * `arena` is a DEVICE buffer of at least *arena_bytes_needed bytes (call with arena == NULL to get
+ * the size: returns GSWA_ERR_WORKSPACE and fills arena_bytes_needed). b_qkv / b_proj may be NULL. */
+int gswa_step_host(const gswa_desc* desc, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
+                   const void* b_proj, const void* bias_table, const void* dy, void* y, void* dx, float* dw_qkv,
+                   float* db_qkv, float* dw_proj, float* db_proj, float* dbias_table, void* arena,
+                   size_t arena_bytes, size_t* arena_bytes_needed, void* cuda_stream);
+
+/* Number of kernels this library has launched in the calling process since load (monotonic). */
+uint64_t gswa_launch_count(void);
+
+/* Text for a gswa_status; for GSWA_ERR_CUDA the text of the last CUDA error seen by this thread. */
+const char* gswa_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GSWA_H_ */

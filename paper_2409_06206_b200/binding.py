@@ -1,0 +1,167 @@
+"""ctypes binding of libgswa.so: argument marshalling only, every step runs in the CUDA library.
+
+The functions mirror the C entry points of include/gswa.h one to one.  Tensors
+are torch tensors used purely as device (or pinned host) memory; their
+`data_ptr()` is what crosses the boundary.  There is no CPU fallback: if the
+library cannot be loaded, importing-and-calling raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libgswa.so")
+
+GSWA_F32, GSWA_BF16 = 0, 1
+FLAG_ACCUMULATE, FLAG_GENERIC = 1, 2
+
+EXPORTS = ("gswa_workspace_query", "gswa_forward", "gswa_backward", "gswa_index_maps", "gswa_step_host",
+           "gswa_launch_count", "gswa_status_string")
+
+
+class GswaError(RuntimeError):
+    def __init__(self, status: int, text: str):
+        super().__init__("libgswa status %d: %s" % (status, text))
+        self.status = status
+
+
+class _Desc(C.Structure):
+    _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("W", C.c_int32), ("C", C.c_int32), ("num_heads", C.c_int32),
+                ("window", C.c_int32), ("num_groups", C.c_int32), ("group_heads", C.POINTER(C.c_int32)),
+                ("group_shift", C.POINTER(C.c_int32)), ("dtype", C.c_int32), ("qk_dim", C.c_int32),
+                ("v_dim", C.c_int32), ("flags", C.c_uint32)]
+
+
+class Desc:
+    """Owns a gswa_desc and the two host arrays it points to."""
+
+    def __init__(self, B: int, H: int, W: int, C_: int, num_heads: int, window: int, group_heads: Sequence[int],
+                 group_shift: Sequence[int], dtype: str = "bf16", flags: int = 0, qk_dim: int = 0, v_dim: int = 0):
+        if len(group_heads) != len(group_shift):
+            raise ValueError("group_heads and group_shift differ in length")
+        G = len(group_heads)
+        self._gh = (C.c_int32 * max(G, 1))(*group_heads)
+        self._gs = (C.c_int32 * max(G, 1))(*group_shift)
+        self.c = _Desc(B, H, W, C_, num_heads, window, G, C.cast(self._gh, C.POINTER(C.c_int32)),
+                       C.cast(self._gs, C.POINTER(C.c_int32)), {"f32": GSWA_F32, "bf16": GSWA_BF16}[dtype], qk_dim,
+                       v_dim, flags)
+        self.dtype = dtype
+        self.shape = (B, H, W, C_)
+        self.num_heads, self.window = num_heads, window
+
+    @classmethod
+    def from_config(cls, cfg, layer: int = 0, batch: Optional[int] = None, flags: int = 0) -> "Desc":
+        from .inputs import layer_groups
+        gh, gs = layer_groups(cfg, layer)
+        return cls(cfg.B if batch is None else batch, cfg.H, cfg.W, cfg.C, cfg.num_heads, cfg.window, gh, gs,
+                   cfg.dtype, flags)
+
+    def with_flags(self, flags: int) -> "Desc":
+        B, H, W, C_ = self.shape
+        return Desc(B, H, W, C_, self.num_heads, self.window, list(self._gh)[:self.c.num_groups],
+                    list(self._gs)[:self.c.num_groups], self.dtype, flags, self.c.qk_dim, self.c.v_dim)
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libgswa.so (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libgswa.so is missing: build it with `python -m paper_2409_06206_b200.build` "
+                               "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, sz, dp = C.c_void_p, C.c_size_t, C.POINTER(_Desc)
+        szp = C.POINTER(C.c_size_t)
+        L.gswa_workspace_query.argtypes = [dp, szp, szp, szp, szp]
+        L.gswa_forward.argtypes = [dp] + [vp] * 9 + [sz, vp]
+        L.gswa_backward.argtypes = [dp] + [vp] * 14 + [sz, vp]
+        L.gswa_index_maps.argtypes = [dp, C.c_int32] + [vp] * 6
+        L.gswa_step_host.argtypes = [dp] + [vp] * 15 + [sz, szp, vp]
+        L.gswa_launch_count.argtypes = []
+        L.gswa_launch_count.restype = C.c_uint64
+        L.gswa_status_string.argtypes = [C.c_int]
+        L.gswa_status_string.restype = C.c_char_p
+        for name in ("gswa_workspace_query", "gswa_forward", "gswa_backward", "gswa_index_maps", "gswa_step_host"):
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+def gswa_status_string(status: int) -> str:
+    return lib().gswa_status_string(int(status)).decode()
+
+
+def _check(status: int) -> None:
+    if status != 0:
+        raise GswaError(status, gswa_status_string(status))
+
+
+def gswa_workspace_query(desc: Desc):
+    """-> (saved_bytes, fwd_scratch_bytes, infer_scratch_bytes, bwd_scratch_bytes)"""
+    out = [C.c_size_t(0) for _ in range(4)]
+    _check(lib().gswa_workspace_query(C.byref(desc.c), *[C.byref(o) for o in out]))
+    return tuple(int(o.value) for o in out)
+
+
+def gswa_forward(desc: Desc, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, y, saved, scratch, scratch_bytes=None,
+                 stream=None) -> None:
+    if scratch_bytes is None:
+        scratch_bytes = 0 if scratch is None else scratch.numel() * scratch.element_size()
+    _check(lib().gswa_forward(C.byref(desc.c), _ptr(x), _ptr(w_qkv), _ptr(b_qkv), _ptr(w_proj), _ptr(b_proj),
+                              _ptr(bias_table), _ptr(y), _ptr(saved), _ptr(scratch), scratch_bytes, _stream(stream)))
+
+
+def gswa_backward(desc: Desc, x, w_qkv, b_qkv, w_proj, bias_table, saved, dy, dx, dw_qkv, db_qkv, dw_proj, db_proj,
+                  dbias_table, scratch, scratch_bytes=None, stream=None) -> None:
+    if scratch_bytes is None:
+        scratch_bytes = 0 if scratch is None else scratch.numel() * scratch.element_size()
+    _check(lib().gswa_backward(C.byref(desc.c), _ptr(x), _ptr(w_qkv), _ptr(b_qkv), _ptr(w_proj), _ptr(bias_table),
+                               _ptr(saved), _ptr(dy), _ptr(dx), _ptr(dw_qkv), _ptr(db_qkv), _ptr(dw_proj),
+                               _ptr(db_proj), _ptr(dbias_table), _ptr(scratch), scratch_bytes, _stream(stream)))
+
+
+def gswa_index_maps(desc: Desc, group: int, win, slot, region, token_of, rel_index, stream=None) -> None:
+    _check(lib().gswa_index_maps(C.byref(desc.c), group, _ptr(win), _ptr(slot), _ptr(region), _ptr(token_of),
+                                 _ptr(rel_index), _stream(stream)))
+
+
+def gswa_step_host_arena_bytes(desc: Desc) -> int:
+    need = C.c_size_t(0)
+    lib().gswa_step_host(C.byref(desc.c), *([None] * 15), 0, C.byref(need), None)
+    return int(need.value)
+
+
+def gswa_step_host(desc: Desc, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, dy, y, dx, dw_qkv, db_qkv, dw_proj,
+                   db_proj, dbias_table, arena, stream=None) -> None:
+    """All tensors except `arena` are HOST tensors (pinned for asynchronous copies)."""
+    need = C.c_size_t(0)
+    _check(lib().gswa_step_host(C.byref(desc.c), _ptr(x), _ptr(w_qkv), _ptr(b_qkv), _ptr(w_proj), _ptr(b_proj),
+                                _ptr(bias_table), _ptr(dy), _ptr(y), _ptr(dx), _ptr(dw_qkv), _ptr(db_qkv),
+                                _ptr(dw_proj), _ptr(db_proj), _ptr(dbias_table), _ptr(arena),
+                                arena.numel() * arena.element_size(), C.byref(need), _stream(stream)))
+
+
+def gswa_launch_count() -> int:
+    return int(lib().gswa_launch_count())

@@ -1,0 +1,222 @@
+// Host side of libgswa: descriptor validation, buffer planning and the extern "C" entry points.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+
+#include "gswa_internal.h"
+
+namespace gswa {
+
+static std::atomic<uint64_t> g_launches{0};
+static thread_local char g_cuda_msg[256] = "no CUDA error recorded";
+
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+int check_launch() {
+  const cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) return GSWA_OK;
+  snprintf(g_cuda_msg, sizeof(g_cuda_msg), "CUDA error: %s", cudaGetErrorString(e));
+  return GSWA_ERR_CUDA;
+}
+
+static int cuda_rc(cudaError_t e) {
+  if (e == cudaSuccess) return GSWA_OK;
+  snprintf(g_cuda_msg, sizeof(g_cuda_msg), "CUDA error: %s", cudaGetErrorString(e));
+  (void)cudaGetLastError();
+  return GSWA_ERR_CUDA;
+}
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+int make_plan(const gswa_desc* desc, Plan* p) {
+  if (desc == nullptr || p == nullptr) return GSWA_ERR_NULL;
+  if (desc->group_heads == nullptr || desc->group_shift == nullptr) return GSWA_ERR_NULL;
+  memset(p, 0, sizeof(*p));
+  p->B = desc->B; p->H = desc->H; p->W = desc->W; p->C = desc->C;
+  p->nh = desc->num_heads; p->M = desc->window; p->G = desc->num_groups;
+  p->dtype = desc->dtype; p->flags = desc->flags;
+  if (p->B < 0 || p->H <= 0 || p->W <= 0 || p->C <= 0 || p->nh <= 0 || p->M <= 0 || p->G <= 0) return GSWA_ERR_SHAPE;
+  if (p->G > kMaxGroups || p->nh > kMaxHeads) return GSWA_ERR_UNSUPPORTED;
+  if (p->C % p->nh != 0 || p->H % p->M != 0 || p->W % p->M != 0) return GSWA_ERR_SHAPE;
+  if (p->dtype != GSWA_F32 && p->dtype != GSWA_BF16) return GSWA_ERR_UNSUPPORTED;
+  p->d = p->C / p->nh;
+  p->N = p->M * p->M;
+  int sum = 0;
+  for (int g = 0; g < p->G; ++g) {
+    p->gh[g] = desc->group_heads[g];
+    p->gs[g] = desc->group_shift[g];
+    p->gh0[g] = sum;
+    if (p->gh[g] <= 0 || p->gs[g] < 0 || p->gs[g] >= p->M) return GSWA_ERR_SHAPE;
+    sum += p->gh[g];
+  }
+  if (sum != p->nh) return GSWA_ERR_SHAPE;
+  if ((desc->qk_dim != 0 && desc->qk_dim != p->d) || (desc->v_dim != 0 && desc->v_dim != p->d))
+    return GSWA_ERR_UNSUPPORTED;
+  if (p->N > 144 || p->d > 64) return GSWA_ERR_UNSUPPORTED;
+  const long long T = (long long)p->B * p->H * p->W;
+  if (T * 3 * p->C >= (1LL << 40) || T >= (1LL << 31) / 2) return GSWA_ERR_UNSUPPORTED;
+  p->T = T;
+  p->nWh = p->H / p->M; p->nWw = p->W / p->M; p->nW = p->nWh * p->nWw;
+  p->esize = p->dtype == GSWA_F32 ? 4 : 2;
+  p->fast = 0;
+  // generic path: saved = qkv[T,3C] | A[T,C] | L[T,nh] (float)
+  const size_t es = (size_t)p->esize;
+  p->off_qkv = 0;
+  p->off_A = align_up((size_t)T * 3 * p->C * es, 256);
+  p->off_L = p->off_A + align_up((size_t)T * p->C * es, 256);
+  p->saved_bytes = p->off_L + align_up((size_t)T * p->nh * sizeof(float), 256);
+  p->fwd_scratch = 0;
+  p->infer_scratch = p->saved_bytes;
+  p->bwd_scratch = align_up((size_t)T * 4 * p->C * es, 256);  // dA[T,C] | dqkv[T,3C]
+  return GSWA_OK;
+}
+
+static bool misaligned(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) != 0; }
+
+}  // namespace gswa
+
+using namespace gswa;
+
+extern "C" {
+
+int gswa_workspace_query(const gswa_desc* desc, size_t* saved_bytes, size_t* fwd_scratch_bytes,
+                         size_t* infer_scratch_bytes, size_t* bwd_scratch_bytes) {
+  Plan p;
+  const int rc = make_plan(desc, &p);
+  if (rc) return rc;
+  if (saved_bytes) *saved_bytes = p.saved_bytes;
+  if (fwd_scratch_bytes) *fwd_scratch_bytes = p.fwd_scratch;
+  if (infer_scratch_bytes) *infer_scratch_bytes = p.infer_scratch;
+  if (bwd_scratch_bytes) *bwd_scratch_bytes = p.bwd_scratch;
+  return GSWA_OK;
+}
+
+int gswa_forward(const gswa_desc* desc, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
+                 const void* b_proj, const void* bias_table, void* y, void* saved, void* scratch,
+                 size_t scratch_bytes, void* cuda_stream) {
+  Plan p;
+  int rc = make_plan(desc, &p);
+  if (rc) return rc;
+  if (!x || !w_qkv || !w_proj || !bias_table || !y) return GSWA_ERR_NULL;
+  const size_t need = saved ? p.fwd_scratch : p.infer_scratch;
+  if (need > 0 && scratch == nullptr) return GSWA_ERR_NULL;
+  if (misaligned(x) || misaligned(w_qkv) || misaligned(b_qkv) || misaligned(w_proj) || misaligned(b_proj) ||
+      misaligned(bias_table) || misaligned(y) || misaligned(saved) || misaligned(scratch))
+    return GSWA_ERR_ALIGN;
+  if (scratch_bytes < need) return GSWA_ERR_WORKSPACE;
+  if (p.T == 0) return GSWA_OK;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  void* carry = saved ? saved : scratch;
+  return generic_forward(p, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, y, carry, st);
+}
+
+int gswa_backward(const gswa_desc* desc, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
+                  const void* bias_table, const void* saved, const void* dy, void* dx, float* dw_qkv,
+                  float* db_qkv, float* dw_proj, float* db_proj, float* dbias_table, void* scratch,
+                  size_t scratch_bytes, void* cuda_stream) {
+  (void)b_qkv;
+  Plan p;
+  int rc = make_plan(desc, &p);
+  if (rc) return rc;
+  if (!x || !w_qkv || !w_proj || !bias_table || !saved || !dy) return GSWA_ERR_NULL;
+  if (p.bwd_scratch > 0 && scratch == nullptr) return GSWA_ERR_NULL;
+  if (misaligned(x) || misaligned(w_qkv) || misaligned(w_proj) || misaligned(bias_table) || misaligned(saved) ||
+      misaligned(dy) || misaligned(dx) || misaligned(dw_qkv) || misaligned(db_qkv) || misaligned(dw_proj) ||
+      misaligned(db_proj) || misaligned(dbias_table) || misaligned(scratch))
+    return GSWA_ERR_ALIGN;
+  if (scratch_bytes < p.bwd_scratch) return GSWA_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (!(p.flags & GSWA_FLAG_ACCUMULATE)) {
+    const size_t C = (size_t)p.C, nrel = (size_t)(2 * p.M - 1) * (2 * p.M - 1);
+    if (dw_qkv && (rc = cuda_rc(cudaMemsetAsync(dw_qkv, 0, 3 * C * C * sizeof(float), st)))) return rc;
+    if (db_qkv && (rc = cuda_rc(cudaMemsetAsync(db_qkv, 0, 3 * C * sizeof(float), st)))) return rc;
+    if (dw_proj && (rc = cuda_rc(cudaMemsetAsync(dw_proj, 0, C * C * sizeof(float), st)))) return rc;
+    if (db_proj && (rc = cuda_rc(cudaMemsetAsync(db_proj, 0, C * sizeof(float), st)))) return rc;
+    if (dbias_table && (rc = cuda_rc(cudaMemsetAsync(dbias_table, 0, nrel * p.nh * sizeof(float), st)))) return rc;
+  }
+  if (p.T == 0) return GSWA_OK;
+  return generic_backward(p, x, w_qkv, w_proj, bias_table, saved, dy, dx, dw_qkv, db_qkv, dw_proj, db_proj,
+                          dbias_table, scratch, st);
+}
+
+int gswa_index_maps(const gswa_desc* desc, int32_t group, int32_t* win, int32_t* slot, int32_t* region,
+                    int32_t* token_of, int32_t* rel_index, void* cuda_stream) {
+  Plan p;
+  const int rc = make_plan(desc, &p);
+  if (rc) return rc;
+  if (group < 0 || group >= p.G) return GSWA_ERR_SHAPE;
+  return launch_index_maps(p, group, win, slot, region, token_of, rel_index, reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int gswa_step_host(const gswa_desc* desc, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
+                   const void* b_proj, const void* bias_table, const void* dy, void* y, void* dx, float* dw_qkv,
+                   float* db_qkv, float* dw_proj, float* db_proj, float* dbias_table, void* arena,
+                   size_t arena_bytes, size_t* arena_bytes_needed, void* cuda_stream) {
+  Plan p;
+  int rc = make_plan(desc, &p);
+  if (rc) return rc;
+  const size_t es = (size_t)p.esize, C = (size_t)p.C, nrel = (size_t)(2 * p.M - 1) * (2 * p.M - 1);
+  const size_t act = align_up((size_t)p.T * C * es, 256);
+  // arena layout
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
+  const size_t o_x = take(act), o_dy = take(act), o_y = take(act), o_dx = take(act);
+  const size_t o_wqkv = take(3 * C * C * es), o_bqkv = take(3 * C * es), o_wproj = take(C * C * es);
+  const size_t o_bproj = take(C * es), o_tab = take(nrel * p.nh * es);
+  const size_t o_dwqkv = take(3 * C * C * 4), o_dbqkv = take(3 * C * 4), o_dwproj = take(C * C * 4);
+  const size_t o_dbproj = take(C * 4), o_dtab = take(nrel * p.nh * 4);
+  const size_t o_saved = take(p.saved_bytes);
+  const size_t scr = p.fwd_scratch > p.bwd_scratch ? p.fwd_scratch : p.bwd_scratch;
+  const size_t o_scr = take(scr);
+  if (arena_bytes_needed) *arena_bytes_needed = off;
+  if (arena == nullptr || arena_bytes < off) return GSWA_ERR_WORKSPACE;
+  if (!x || !w_qkv || !w_proj || !bias_table || !dy || !y || !dx || !dw_qkv || !db_qkv || !dw_proj || !db_proj ||
+      !dbias_table)
+    return GSWA_ERR_NULL;
+  if (misaligned(arena)) return GSWA_ERR_ALIGN;
+  char* a = static_cast<char*>(arena);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const size_t act_b = (size_t)p.T * C * es;
+  auto h2d = [&](size_t o, const void* src, size_t bytes) {
+    return cuda_rc(cudaMemcpyAsync(a + o, src, bytes, cudaMemcpyHostToDevice, st));
+  };
+  auto d2h = [&](void* dst, size_t o, size_t bytes) {
+    return cuda_rc(cudaMemcpyAsync(dst, a + o, bytes, cudaMemcpyDeviceToHost, st));
+  };
+  if ((rc = h2d(o_x, x, act_b)) || (rc = h2d(o_dy, dy, act_b)) || (rc = h2d(o_wqkv, w_qkv, 3 * C * C * es)) ||
+      (rc = h2d(o_wproj, w_proj, C * C * es)) || (rc = h2d(o_tab, bias_table, nrel * p.nh * es)))
+    return rc;
+  if (b_qkv && (rc = h2d(o_bqkv, b_qkv, 3 * C * es))) return rc;
+  if (b_proj && (rc = h2d(o_bproj, b_proj, C * es))) return rc;
+  rc = gswa_forward(desc, a + o_x, a + o_wqkv, b_qkv ? a + o_bqkv : nullptr, a + o_wproj, b_proj ? a + o_bproj : nullptr,
+                    a + o_tab, a + o_y, a + o_saved, a + o_scr, scr, cuda_stream);
+  if (rc) return rc;
+  gswa_desc d2 = *desc;
+  d2.flags &= ~GSWA_FLAG_ACCUMULATE;
+  rc = gswa_backward(&d2, a + o_x, a + o_wqkv, b_qkv ? a + o_bqkv : nullptr, a + o_wproj, a + o_tab, a + o_saved,
+                     a + o_dy, a + o_dx, (float*)(a + o_dwqkv), (float*)(a + o_dbqkv), (float*)(a + o_dwproj),
+                     (float*)(a + o_dbproj), (float*)(a + o_dtab), a + o_scr, scr, cuda_stream);
+  if (rc) return rc;
+  if ((rc = d2h(y, o_y, act_b)) || (rc = d2h(dx, o_dx, act_b)) || (rc = d2h(dw_qkv, o_dwqkv, 3 * C * C * 4)) ||
+      (rc = d2h(db_qkv, o_dbqkv, 3 * C * 4)) || (rc = d2h(dw_proj, o_dwproj, C * C * 4)) ||
+      (rc = d2h(db_proj, o_dbproj, C * 4)) || (rc = d2h(dbias_table, o_dtab, nrel * p.nh * 4)))
+    return rc;
+  return cuda_rc(cudaStreamSynchronize(st));
+}
+
+uint64_t gswa_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* gswa_status_string(int status) {
+  switch (status) {
+    case GSWA_OK: return "ok";
+    case GSWA_ERR_NULL: return "a required pointer is NULL";
+    case GSWA_ERR_SHAPE: return "inconsistent layer description";
+    case GSWA_ERR_ALIGN: return "device pointer not 16-byte aligned";
+    case GSWA_ERR_UNSUPPORTED: return "layer description not supported";
+    case GSWA_ERR_WORKSPACE: return "scratch or arena buffer too small";
+    case GSWA_ERR_CUDA: return g_cuda_msg;
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

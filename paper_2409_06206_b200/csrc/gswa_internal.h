@@ -1,0 +1,52 @@
+// Internal declarations shared by the host planner and the kernel files of libgswa.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "gswa.h"
+
+namespace gswa {
+
+constexpr int kMaxGroups = 16;
+constexpr int kMaxHeads = 64;
+
+// Validated, flattened copy of a gswa_desc plus derived sizes.
+struct Plan {
+  int B, H, W, C, nh, d, M, N, G;
+  int nWh, nWw, nW;            // windows per image: rows, cols, total
+  long long T;                 // tokens = B*H*W
+  int dtype;
+  uint32_t flags;
+  int gh[kMaxGroups], gs[kMaxGroups], gh0[kMaxGroups];  // heads, shift, first head of each group
+  int esize;                   // bytes per element of dtype
+  int fast;                    // 1 = bf16 tensor-core path, 0 = generic CUDA-core path
+  // fast-path geometry
+  int dp;                      // head dim padded to an MMA-friendly width (16 or 32)
+  int Cp;                      // C padded to a multiple of 64 (GEMM K / row pitch of padded activations)
+  // byte offsets inside `saved`
+  size_t off_qkv, off_A, off_L, saved_bytes;
+  size_t fwd_scratch, infer_scratch, bwd_scratch;
+};
+
+// Per-head shift table passed by value to the attention kernels.
+struct HeadShifts {
+  int8_t s[kMaxHeads];
+};
+
+int make_plan(const gswa_desc* desc, Plan* plan);
+void count_launch(int n = 1);
+int check_launch();  // GSWA_OK or GSWA_ERR_CUDA (records the CUDA error text)
+
+// ---- generic CUDA-core path (any shape the descriptor allows, f32 or bf16 storage, f32 arithmetic)
+int generic_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
+                    const void* b_proj, const void* table, void* y, void* saved, cudaStream_t st);
+int generic_backward(const Plan& p, const void* x, const void* w_qkv, const void* w_proj, const void* table,
+                     const void* saved, const void* dy, void* dx, float* dw_qkv, float* db_qkv, float* dw_proj,
+                     float* db_proj, float* dtable, void* scratch, cudaStream_t st);
+int launch_index_maps(const Plan& p, int group, int32_t* win, int32_t* slot, int32_t* region, int32_t* token_of,
+                      int32_t* rel, cudaStream_t st);
+
+}  // namespace gswa

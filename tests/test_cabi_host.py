@@ -1,0 +1,69 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports what include/gswa.h
+declares, validates descriptors and reports errors before anything is enqueued."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2409_06206_b200 import binding as gb
+from paper_2409_06206_b200 import build as gbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    gbuild.build()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "gswa.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(gswa_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = _declared()
+    assert set(gb.EXPORTS) <= set(names)
+    L = ctypes.CDLL(gb.LIB_PATH)
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_workspace_query_and_descriptor_validation():
+    d = gb.Desc(2, 16, 16, 60, 6, 8, (3, 3), (0, 4), "f32")
+    saved, fwd, infer, bwd = gb.gswa_workspace_query(d)
+    assert saved > 0 and infer >= saved - 1 and bwd > 0 and fwd >= 0
+    bad = [
+        (gb.Desc(1, 12, 16, 60, 6, 8, (3, 3), (0, 4)), -2),       # H not a multiple of M
+        (gb.Desc(1, 16, 16, 60, 6, 8, (3, 2), (0, 4)), -2),       # heads do not add up
+        (gb.Desc(1, 16, 16, 60, 6, 8, (3, 3), (0, 8)), -2),       # shift out of range
+        (gb.Desc(1, 16, 16, 62, 6, 8, (3, 3), (0, 4)), -2),       # C not divisible by heads
+        (gb.Desc(1, 16, 16, 60, 6, 8, (3, 3), (0, 4), qk_dim=16), -4),
+        (gb.Desc(1, 16, 16, 60, 6, 8, (), ()), -2),
+    ]
+    for desc, code in bad:
+        with pytest.raises(gb.GswaError) as e:
+            gb.gswa_workspace_query(desc)
+        assert e.value.status == code, (desc.shape, e.value.status)
+
+
+def test_argument_errors_are_reported_before_any_launch():
+    d = gb.Desc(1, 16, 16, 60, 6, 8, (3, 3), (0, 4), "f32")
+    n0 = gb.gswa_launch_count()
+    with pytest.raises(gb.GswaError) as e:
+        gb.gswa_forward(d, None, 256, None, 256, None, 256, 256, 256, 256, 1 << 30, stream=0)
+    assert e.value.status == -1
+    with pytest.raises(gb.GswaError) as e:                       # misaligned x
+        gb.gswa_forward(d, 264, 256, None, 256, None, 256, 256, 256, 256, 1 << 30, stream=0)
+    assert e.value.status == -3
+    with pytest.raises(gb.GswaError) as e:                       # inference scratch too small
+        gb.gswa_forward(d, 256, 256, None, 256, None, 256, 256, None, 256, 16, stream=0)
+    assert e.value.status == -5
+    with pytest.raises(gb.GswaError) as e:                       # backward scratch too small
+        gb.gswa_backward(d, 256, 256, None, 256, 256, 256, 256, 256, 256, 256, 256, 256, 256, 256, 16, stream=0)
+    assert e.value.status == -5
+    assert gb.gswa_launch_count() == n0
+    assert gb.gswa_step_host_arena_bytes(d) > 0
+    assert "NULL" in gb.gswa_status_string(-1) and gb.gswa_status_string(0) == "ok"

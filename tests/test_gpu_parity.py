@@ -1,0 +1,180 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 CPU checker on the same
+seeded inputs.  Index maps must be bit-exact; tensors within 1e-4 (f32) / 2e-2 (bf16) of the checker,
+measured as max |gpu - ref| / max |ref| per tensor."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+from oracle import gswa_oracle as orc
+from paper_2409_06206_b200 import binding as gb
+from paper_2409_06206_b200 import build as gbuild
+from paper_2409_06206_b200.inputs import CONFIGS, LayerConfig, make_inputs
+
+from gpu_util import GRADS, assert_close, rel_err, run_gpu, run_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    gbuild.build()
+
+
+@pytest.mark.parametrize("H,W,M,s", [(16, 16, 8, 4), (16, 24, 8, 3), (64, 64, 8, 4), (8, 8, 8, 7), (24, 12, 4, 1),
+                                     (36, 24, 12, 6), (16, 16, 8, 0)])
+def test_index_maps_bit_exact(H, W, M, s):
+    import torch
+    d = gb.Desc(1, H, W, 12, 2, M, (1, 1), (0, s), "f32")
+    N = M * M
+    bufs = [torch.full((H * W,), -1, dtype=torch.int32, device="cuda") for _ in range(4)]
+    rel = torch.full((N * N,), -1, dtype=torch.int32, device="cuda")
+    gb.gswa_index_maps(d, 1, *bufs, rel)
+    torch.cuda.synchronize()
+    win, slot, region, rel_ref = orc.index_maps(H, W, M, s)
+    got = [b.cpu().numpy() for b in bufs]
+    assert np.array_equal(got[0], win.ravel())
+    assert np.array_equal(got[1], slot.ravel())
+    assert np.array_equal(got[2], region.ravel())
+    token_of = np.empty(H * W, np.int32)
+    token_of[win.ravel() * N + slot.ravel()] = np.arange(H * W, dtype=np.int32)
+    assert np.array_equal(got[3], token_of)
+    assert np.array_equal(rel.cpu().numpy(), rel_ref.ravel())
+
+
+def test_config1_f32_forward_backward():
+    cfg = CONFIGS["c1"]
+    inp = make_inputs(cfg)
+    got = run_gpu(cfg, inp)
+    ref = run_oracle(cfg, inp)
+    errs = assert_close(got, ref, "f32")
+    assert set(errs) == set(GRADS) | {"y"}
+
+
+def _mk(name, B, H, W, C, nh, M, gh, gs, dtype, seed=1):
+    return LayerConfig(name, B, H, W, C, nh, M, gh, gs, dtype=dtype, seed=seed, bias_std=0.1)
+
+
+SWEEP = [
+    _mk("s0", 2, 8, 8, 12, 2, 8, (2,), (0,), "f32"),
+    _mk("s1", 1, 8, 8, 12, 2, 8, (1, 1), (3, 7), "f32"),
+    _mk("s2", 2, 16, 24, 60, 6, 8, (3, 3), (0, 4), "f32"),
+    _mk("s3", 1, 24, 16, 60, 6, 8, (1, 2, 3), (1, 0, 5), "f32"),
+    _mk("s4", 2, 16, 16, 180, 6, 8, (3, 3), (4, 0), "f32"),
+    _mk("s5", 1, 24, 24, 24, 2, 12, (1, 1), (0, 6), "f32"),
+    _mk("s6", 3, 12, 8, 16, 4, 4, (2, 2), (0, 2), "f32"),
+    _mk("s7", 2, 16, 24, 60, 6, 8, (3, 3), (0, 4), "bf16"),
+    _mk("s8", 1, 24, 16, 180, 6, 8, (3, 3), (4, 0), "bf16"),
+    _mk("s9", 2, 16, 16, 180, 6, 8, (2, 4), (3, 0), "bf16"),
+    _mk("s10", 3, 24, 40, 60, 6, 8, (6,), (4,), "bf16"),
+    _mk("s11", 5, 16, 16, 64, 2, 8, (1, 1), (0, 1), "bf16"),
+    _mk("s12", 1, 24, 24, 36, 3, 12, (1, 2), (0, 6), "bf16"),
+]
+
+
+@pytest.mark.parametrize("cfg", SWEEP, ids=[c.name for c in SWEEP])
+def test_small_shapes_forward_backward(cfg):
+    inp = make_inputs(cfg)
+    got = run_gpu(cfg, inp)
+    ref = run_oracle(cfg, inp)
+    assert_close(got, ref, cfg.dtype)
+
+
+@pytest.mark.parametrize("cfg", [SWEEP[2], SWEEP[7], SWEEP[8]], ids=["f32", "bf16-c60", "bf16-c180"])
+def test_generic_kernels_forced(cfg):
+    inp = make_inputs(cfg)
+    got = run_gpu(cfg, inp, flags=gb.FLAG_GENERIC)
+    ref = run_oracle(cfg, inp)
+    assert_close(got, ref, cfg.dtype)
+
+
+def test_null_biases_inference_mode_and_accumulate():
+    import torch
+    cfg = dataclasses.replace(SWEEP[7], bias_std=0.0)
+    inp = make_inputs(cfg)
+    ref = run_oracle(cfg, inp)
+    got = run_gpu(cfg, inp, use_bias=False)
+    assert_close(got, ref, cfg.dtype)
+    inf = run_gpu(cfg, inp, inference=True)
+    assert rel_err(inf["y"], got["y"]) == 0.0
+    # accumulate flag: gradients are added to what the buffers hold (run_gpu pre-fills them with 7)
+    acc = run_gpu(cfg, inp, flags=gb.FLAG_ACCUMULATE)
+    for n in GRADS[1:]:
+        assert rel_err(acc[n] - 7.0, ref[n]) <= 2e-2, n
+
+
+def test_empty_batch_is_a_no_op():
+    import torch
+    cfg = SWEEP[7]
+    d = gb.Desc(0, cfg.H, cfg.W, cfg.C, cfg.num_heads, cfg.window, cfg.group_heads, cfg.group_shift, "bf16")
+    t = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    n0 = gb.gswa_launch_count()
+    gb.gswa_forward(d, t, t, None, t, None, t, t, t, t)
+    assert gb.gswa_launch_count() == n0
+
+
+@pytest.mark.parametrize("name,batch", [("c2", 8), ("c3", 4)])
+def test_training_shapes_reduced_batch(name, batch):
+    """The paper-shaped training layers at a batch the checker finishes in seconds (weight gradients included)."""
+    cfg = CONFIGS[name]
+    inp = make_inputs(cfg, batch=batch)
+    got = run_gpu(cfg, inp)
+    ref = run_oracle(cfg, inp, chunk=4)
+    assert_close(got, ref, cfg.dtype)
+
+
+@pytest.mark.parametrize("name", ["cM", "c4"])
+def test_full_size_sampled_images_and_properties(name):
+    """Full-size launch configuration: y and dx of sampled batch items against the checker (batch items are
+    independent), plus properties of the parameter gradients that hold at any size."""
+    cfg = CONFIGS[name]
+    inp = make_inputs(cfg)
+    got = run_gpu(cfg, inp)
+    picks = [0, cfg.B // 2 + 1, cfg.B - 1]
+    sub = {k: (v[picks] if k in ("x", "dy") else v) for k, v in inp.items()}
+    ref = run_oracle(cfg, sub, chunk=3)
+    assert rel_err(got["y"][picks], ref["y"]) <= 2e-2
+    assert rel_err(got["dx"][picks], ref["dx"]) <= 2e-2
+    dy2 = inp["dy"].reshape(-1, cfg.C).astype(np.float64)
+    assert rel_err(got["db_proj"], dy2.sum(0)) <= 2e-2
+    scale = np.abs(got["dbias_table"]).max()
+    assert np.abs(got["dbias_table"].sum(0)).max() <= 2e-2 * scale * 15       # columns sum to 0 (softmax invariance)
+    assert np.abs(got["db_qkv"][cfg.C:2 * cfg.C]).max() <= 2e-2 * np.abs(got["db_qkv"]).max()   # key bias gradient is 0
+    for n in GRADS:
+        assert np.isfinite(got[n]).all()
+
+
+def test_stacked_inference_layers():
+    """Six stacked layers with alternating group assignment on a reduced image; every layer checked."""
+    cfg = dataclasses.replace(CONFIGS["c5"], H=64, W=64)
+    x = make_inputs(cfg, tensors=("x",))["x"]
+    for layer in range(cfg.layers):
+        inp = make_inputs(cfg, layer=layer, tensors=("w_qkv", "b_qkv", "w_proj", "b_proj", "bias_table"))
+        inp["x"] = x
+        got = run_gpu(cfg, inp, backward=False, layer=layer, inference=True)
+        ref = run_oracle(cfg, inp, backward=False, layer=layer)
+        assert rel_err(got["y"], ref["y"]) <= 2e-2
+        from paper_2409_06206_b200.inputs import round_to_bf16
+        x = round_to_bf16(got["y"].astype(np.float32)) * np.float32(4.0)   # keep activations O(1) between layers
+        x = round_to_bf16(x)
+
+
+def test_step_host_matches_device_path():
+    import torch
+    cfg = SWEEP[7]
+    inp = make_inputs(cfg)
+    ref = run_gpu(cfg, inp)
+    desc = gb.Desc.from_config(cfg)
+    tdt = torch.bfloat16
+    host = {k: torch.from_numpy(v).to(tdt).pin_memory() for k, v in inp.items()}
+    C, M, nh = cfg.C, cfg.window, cfg.num_heads
+    out = {"y": torch.empty(inp["x"].shape, dtype=tdt).pin_memory(), "dx": torch.empty(inp["x"].shape, dtype=tdt).pin_memory(),
+           "dw_qkv": torch.empty(3 * C, C).pin_memory(), "db_qkv": torch.empty(3 * C).pin_memory(),
+           "dw_proj": torch.empty(C, C).pin_memory(), "db_proj": torch.empty(C).pin_memory(),
+           "dbias_table": torch.empty((2 * M - 1) ** 2, nh).pin_memory()}
+    arena = torch.empty(gb.gswa_step_host_arena_bytes(desc), dtype=torch.uint8, device="cuda")
+    gb.gswa_step_host(desc, host["x"], host["w_qkv"], host["b_qkv"], host["w_proj"], host["b_proj"], host["bias_table"],
+                      host["dy"], out["y"], out["dx"], out["dw_qkv"], out["db_qkv"], out["dw_proj"], out["db_proj"],
+                      out["dbias_table"], arena)
+    for n, t in out.items():
+        assert rel_err(t.float().numpy().astype(np.float64), ref[n]) <= 1e-3, n
