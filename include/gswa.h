@@ -120,6 +120,13 @@ int gswa_step_host(const gswa_desc* desc, const void* x, const void* w_qkv, cons
                    float* db_qkv, float* dw_proj, float* db_proj, float* dbias_table, void* arena,
                    size_t arena_bytes, size_t* arena_bytes_needed, void* cuda_stream);
 
+/* Per-launch timing for benchmarks (the paper has no counterpart).  While enabled, every kernel the
+ * library launches is bracketed by a CUDA event pair on its stream.  gswa_profile_read waits for the
+ * recorded launches, writes up to max_records entries (names: max_records x 32 chars, NUL-terminated;
+ * ms: milliseconds), stores the number written in *count and clears the list.  Host pointers. */
+int gswa_profile_enable(int on);
+int gswa_profile_read(int32_t max_records, char* names, float* ms, int32_t* count);
+
 /* Number of kernels this library has launched in the calling process since load (monotonic). */
 uint64_t gswa_launch_count(void);
 

@@ -18,7 +18,7 @@ GSWA_F32, GSWA_BF16 = 0, 1
 FLAG_ACCUMULATE, FLAG_GENERIC = 1, 2
 
 EXPORTS = ("gswa_workspace_query", "gswa_forward", "gswa_backward", "gswa_index_maps", "gswa_step_host",
-           "gswa_launch_count", "gswa_status_string")
+           "gswa_profile_enable", "gswa_profile_read", "gswa_launch_count", "gswa_status_string")
 
 
 class GswaError(RuntimeError):
@@ -82,6 +82,10 @@ def lib() -> C.CDLL:
         L.gswa_backward.argtypes = [dp] + [vp] * 14 + [sz, vp]
         L.gswa_index_maps.argtypes = [dp, C.c_int32] + [vp] * 6
         L.gswa_step_host.argtypes = [dp] + [vp] * 15 + [sz, szp, vp]
+        L.gswa_profile_enable.argtypes = [C.c_int]
+        L.gswa_profile_read.argtypes = [C.c_int32, C.c_char_p, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+        L.gswa_profile_enable.restype = C.c_int
+        L.gswa_profile_read.restype = C.c_int
         L.gswa_launch_count.argtypes = []
         L.gswa_launch_count.restype = C.c_uint64
         L.gswa_status_string.argtypes = [C.c_int]
@@ -161,6 +165,20 @@ def gswa_step_host(desc: Desc, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, dy, 
                                 _ptr(bias_table), _ptr(dy), _ptr(y), _ptr(dx), _ptr(dw_qkv), _ptr(db_qkv),
                                 _ptr(dw_proj), _ptr(db_proj), _ptr(dbias_table), _ptr(arena),
                                 arena.numel() * arena.element_size(), C.byref(need), _stream(stream)))
+
+
+def gswa_profile_enable(on: bool) -> None:
+    _check(lib().gswa_profile_enable(1 if on else 0))
+
+
+def gswa_profile_read(max_records: int = 4096):
+    """-> list of (kernel name, milliseconds), one entry per launch recorded since the last read."""
+    names = C.create_string_buffer(max_records * 32)
+    ms = (C.c_float * max_records)()
+    n = C.c_int32(0)
+    _check(lib().gswa_profile_read(max_records, names, ms, C.byref(n)))
+    raw = names.raw
+    return [(raw[i * 32:(i + 1) * 32].split(b"\0", 1)[0].decode(), float(ms[i])) for i in range(n.value)]
 
 
 def gswa_launch_count() -> int:

@@ -1,5 +1,7 @@
 // Host side of libgswa: descriptor validation, buffer planning and the extern "C" entry points.
 #include <atomic>
+#include <mutex>
+#include <vector>
 #include <cstdio>
 #include <cstring>
 
@@ -10,7 +12,31 @@ namespace gswa {
 static std::atomic<uint64_t> g_launches{0};
 static thread_local char g_cuda_msg[256] = "no CUDA error recorded";
 
-void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+// ---- optional per-launch timing (gswa_profile_enable / gswa_profile_read)
+struct ProfRecord {
+  const char* name;
+  cudaEvent_t e0, e1;
+};
+static std::mutex g_prof_mu;
+static bool g_prof_on = false;
+static std::vector<ProfRecord> g_prof;
+
+KernelScope::KernelScope(const char* name, cudaStream_t s) : st(s), slot(-1) {
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (!g_prof_on) return;
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  ProfRecord r{name, nullptr, nullptr};
+  if (cudaEventCreate(&r.e0) != cudaSuccess || cudaEventCreate(&r.e1) != cudaSuccess) return;
+  cudaEventRecord(r.e0, st);
+  g_prof.push_back(r);
+  slot = (int)g_prof.size() - 1;
+}
+
+KernelScope::~KernelScope() {
+  if (slot < 0) return;
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  if (slot < (int)g_prof.size()) cudaEventRecord(g_prof[slot].e1, st);
+}
 
 int check_launch() {
   const cudaError_t e = cudaGetLastError();
@@ -202,6 +228,34 @@ int gswa_step_host(const gswa_desc* desc, const void* x, const void* w_qkv, cons
       (rc = d2h(db_proj, o_dbproj, C * 4)) || (rc = d2h(dbias_table, o_dtab, nrel * p.nh * 4)))
     return rc;
   return cuda_rc(cudaStreamSynchronize(st));
+}
+
+int gswa_profile_enable(int on) {
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  g_prof_on = on != 0;
+  return GSWA_OK;
+}
+
+int gswa_profile_read(int32_t max_records, char* names, float* ms, int32_t* count) {
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  int n = 0, rc = GSWA_OK;
+  for (auto& r : g_prof) {
+    float t = 0.f;
+    if (cudaEventSynchronize(r.e1) != cudaSuccess || cudaEventElapsedTime(&t, r.e0, r.e1) != cudaSuccess) {
+      rc = cuda_rc(cudaGetLastError());
+      if (rc == GSWA_OK) rc = GSWA_ERR_CUDA;
+    }
+    if (n < max_records && names && ms) {
+      snprintf(names + (size_t)n * 32, 32, "%s", r.name);
+      ms[n] = t;
+      ++n;
+    }
+    cudaEventDestroy(r.e0);
+    cudaEventDestroy(r.e1);
+  }
+  g_prof.clear();
+  if (count) *count = n;
+  return rc;
 }
 
 uint64_t gswa_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

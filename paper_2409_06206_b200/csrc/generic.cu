@@ -290,9 +290,8 @@ int launch_gemm(const TA* A, long long sam, long long sak, const TB* Bm, long lo
                 long long scm, const TB* bias, long long Mr, int Nc, long long K, float scale, int scale_cols,
                 cudaStream_t st) {
   dim3 grid((unsigned)((Mr + GB - 1) / GB), (Nc + GB - 1) / GB, 1);
-  gemm_generic<TA, TB, TC, false><<<grid, 256, 0, st>>>(A, sam, sak, Bm, sbk, sbn, Cm, scm, bias, (int)Mr, Nc, K, K,
-                                                        scale, scale_cols);
-  count_launch();
+  { KernelScope ks_("gemm_generic", st); gemm_generic<TA, TB, TC, false><<<grid, 256, 0, st>>>(A, sam, sak, Bm, sbk, sbn, Cm, scm, bias, (int)Mr, Nc, K, K,
+                                                        scale, scale_cols); }
   return check_launch();
 }
 
@@ -306,9 +305,8 @@ int launch_gemm_tn(const TA* G, long long ldg, int n1, const TB* X, long long ld
   long long kchunk = ((rows + splits - 1) / splits + GK - 1) / GK * GK;
   splits = (rows + kchunk - 1) / kchunk;
   dim3 grid((n1 + GB - 1) / GB, (n2 + GB - 1) / GB, (unsigned)splits);
-  gemm_generic<TA, TB, float, true><<<grid, 256, 0, st>>>(G, 1, ldg, X, ldx, 1, Cm, n2, nullptr, n1, n2, rows, kchunk,
-                                                          1.f, 0);
-  count_launch();
+  { KernelScope ks_("gemm_tn_generic", st); gemm_generic<TA, TB, float, true><<<grid, 256, 0, st>>>(G, 1, ldg, X, ldx, 1, Cm, n2, nullptr, n1, n2, rows, kchunk,
+                                                          1.f, 0); }
   return check_launch();
 }
 
@@ -318,8 +316,7 @@ int launch_colsum(const T* G, long long rows, int cols, long long ld, float* out
   if (chunks > 2048) chunks = 2048;
   const long long rchunk = (rows + chunks - 1) / chunks;
   dim3 grid((cols + 31) / 32, (unsigned)chunks);
-  colsum_generic<T><<<grid, 256, 0, st>>>(G, rows, cols, ld, rchunk, out);
-  count_launch();
+  { KernelScope ks_("colsum_generic", st); colsum_generic<T><<<grid, 256, 0, st>>>(G, rows, cols, ld, rchunk, out); }
   return check_launch();
 }
 
@@ -350,8 +347,7 @@ int forward_t(const Plan& p, const T* x, const T* w_qkv, const T* b_qkv, const T
   const size_t smem = attn_fwd_smem(p);
   if (cudaFuncSetAttribute(attn_fwd_generic<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return check_launch();
-  attn_fwd_generic<T><<<dim3(p.B * p.nW, p.nh), 128, smem, st>>>(g, head_shifts(p), qkv, table, A, L);
-  count_launch();
+  { KernelScope ks_("attn_fwd_generic", st); attn_fwd_generic<T><<<dim3(p.B * p.nW, p.nh), 128, smem, st>>>(g, head_shifts(p), qkv, table, A, L); }
   if ((rc = check_launch())) return rc;
   return launch_gemm<T, T, T>(A, C, 1, w_proj, 1, C, y, C, b_proj, p.T, C, C, 1.f, 0, st);
 }
@@ -376,9 +372,8 @@ int backward_t(const Plan& p, const T* x, const T* w_qkv, const T* w_proj, const
   const size_t smem = attn_bwd_smem(p);
   if (cudaFuncSetAttribute(attn_bwd_generic<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return check_launch();
-  attn_bwd_generic<T><<<dim3(p.B * p.nW, p.nh), 256, smem, st>>>(g, head_shifts(p), scale, qkv, table, A, L, dA, dqkv,
-                                                                 dtable);
-  count_launch();
+  { KernelScope ks_("attn_bwd_generic", st); attn_bwd_generic<T><<<dim3(p.B * p.nW, p.nh), 256, smem, st>>>(g, head_shifts(p), scale, qkv, table, A, L, dA, dqkv,
+                                                                 dtable); }
   if ((rc = check_launch())) return rc;
   if (dx && (rc = launch_gemm<T, T, T>(dqkv, 3 * C, 1, w_qkv, C, 1, dx, C, nullptr, p.T, C, 3 * C, 1.f, 0, st)))
     return rc;
@@ -414,8 +409,7 @@ int generic_backward(const Plan& p, const void* x, const void* w_qkv, const void
 int launch_index_maps(const Plan& p, int group, int32_t* win, int32_t* slot, int32_t* region, int32_t* token_of,
                       int32_t* rel, cudaStream_t st) {
   const int n = max(p.H * p.W, p.N * p.N);
-  index_maps_kernel<<<(n + 255) / 256, 256, 0, st>>>(p.H, p.W, p.M, p.gs[group], win, slot, region, token_of, rel);
-  count_launch();
+  { KernelScope ks_("index_maps", st); index_maps_kernel<<<(n + 255) / 256, 256, 0, st>>>(p.H, p.W, p.M, p.gs[group], win, slot, region, token_of, rel); }
   return check_launch();
 }
 

@@ -37,8 +37,16 @@ struct HeadShifts {
 };
 
 int make_plan(const gswa_desc* desc, Plan* plan);
-void count_launch(int n = 1);
 int check_launch();  // GSWA_OK or GSWA_ERR_CUDA (records the CUDA error text)
+
+// Wraps one kernel launch: counts it and, while profiling is enabled, brackets it with a CUDA
+// event pair on the launching stream.  Usage: { KernelScope k("name", st); kernel<<<...>>>(...); }
+struct KernelScope {
+  KernelScope(const char* name, cudaStream_t st);
+  ~KernelScope();
+  cudaStream_t st;
+  int slot;
+};
 
 // ---- generic CUDA-core path (any shape the descriptor allows, f32 or bf16 storage, f32 arithmetic)
 int generic_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
