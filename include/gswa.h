@@ -48,7 +48,8 @@ typedef enum gswa_status {
   GSWA_ERR_ALIGN = -3,       /* a device pointer is not 16-byte aligned                     */
   GSWA_ERR_UNSUPPORTED = -4, /* valid but not implemented (e.g. qk_dim != head_dim)         */
   GSWA_ERR_WORKSPACE = -5,   /* scratch / saved buffer too small                            */
-  GSWA_ERR_CUDA = -6         /* a CUDA runtime call or launch failed                        */
+  GSWA_ERR_CUDA = -6,        /* a CUDA runtime call or launch failed                        */
+  GSWA_ERR_DEVICE = -7       /* a kernel gave up on a bounded internal wait (gswa_scratch_status) */
 } gswa_status;
 
 enum { GSWA_F32 = 0, GSWA_BF16 = 1 };
@@ -119,6 +120,13 @@ int gswa_step_host(const gswa_desc* desc, const void* x, const void* w_qkv, cons
                    const void* b_proj, const void* bias_table, const void* dy, void* y, void* dx, float* dw_qkv,
                    float* db_qkv, float* dw_proj, float* db_proj, float* dbias_table, void* arena,
                    size_t arena_bytes, size_t* arena_bytes_needed, void* cuda_stream);
+
+/* Device-side status of the last gswa_forward / gswa_backward that used `scratch` (the paper has no
+ * counterpart).  The tensor-core kernels hand tiles between warps through barriers whose waits are
+ * bounded; a wait that runs out makes the kernel return early and set a word at the start of
+ * `scratch`.  This call waits for `cuda_stream`, reads the word and returns GSWA_OK or
+ * GSWA_ERR_DEVICE (outputs are then invalid; the context stays usable). */
+int gswa_scratch_status(const gswa_desc* desc, const void* scratch, void* cuda_stream);
 
 /* Per-launch timing for benchmarks (the paper has no counterpart).  While enabled, every kernel the
  * library launches is bracketed by a CUDA event pair on its stream.  gswa_profile_read waits for the

@@ -18,7 +18,7 @@ GSWA_F32, GSWA_BF16 = 0, 1
 FLAG_ACCUMULATE, FLAG_GENERIC = 1, 2
 
 EXPORTS = ("gswa_workspace_query", "gswa_forward", "gswa_backward", "gswa_index_maps", "gswa_step_host",
-           "gswa_profile_enable", "gswa_profile_read", "gswa_launch_count", "gswa_status_string")
+           "gswa_scratch_status", "gswa_profile_enable", "gswa_profile_read", "gswa_launch_count", "gswa_status_string")
 
 
 class GswaError(RuntimeError):
@@ -82,6 +82,8 @@ def lib() -> C.CDLL:
         L.gswa_backward.argtypes = [dp] + [vp] * 14 + [sz, vp]
         L.gswa_index_maps.argtypes = [dp, C.c_int32] + [vp] * 6
         L.gswa_step_host.argtypes = [dp] + [vp] * 15 + [sz, szp, vp]
+        L.gswa_scratch_status.argtypes = [dp, vp, vp]
+        L.gswa_scratch_status.restype = C.c_int
         L.gswa_profile_enable.argtypes = [C.c_int]
         L.gswa_profile_read.argtypes = [C.c_int32, C.c_char_p, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
         L.gswa_profile_enable.restype = C.c_int
@@ -165,6 +167,11 @@ def gswa_step_host(desc: Desc, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, dy, 
                                 _ptr(bias_table), _ptr(dy), _ptr(y), _ptr(dx), _ptr(dw_qkv), _ptr(db_qkv),
                                 _ptr(dw_proj), _ptr(db_proj), _ptr(dbias_table), _ptr(arena),
                                 arena.numel() * arena.element_size(), C.byref(need), _stream(stream)))
+
+
+def gswa_scratch_status(desc: Desc, scratch, stream=None) -> None:
+    """Waits for the stream and raises GswaError(-7) if a kernel of the last call on `scratch` gave up a wait."""
+    _check(lib().gswa_scratch_status(C.byref(desc.c), _ptr(scratch), _stream(stream)))
 
 
 def gswa_profile_enable(on: bool) -> None:

@@ -5,6 +5,7 @@
 #include <cstdio>
 #include <cstring>
 
+#include "fast.cuh"
 #include "gswa_internal.h"
 
 namespace gswa {
@@ -94,6 +95,7 @@ int make_plan(const gswa_desc* desc, Plan* p) {
   p->fwd_scratch = 0;
   p->infer_scratch = p->saved_bytes;
   p->bwd_scratch = align_up((size_t)T * 4 * p->C * es, 256);  // dA[T,C] | dqkv[T,3C]
+  if (fast_path_ok(*p)) fast_plan_sizes(p);
   return GSWA_OK;
 }
 
@@ -124,6 +126,7 @@ int gswa_forward(const gswa_desc* desc, const void* x, const void* w_qkv, const 
   int rc = make_plan(desc, &p);
   if (rc) return rc;
   if (!x || !w_qkv || !w_proj || !bias_table || !y) return GSWA_ERR_NULL;
+  if (p.T == 0) return GSWA_OK;
   const size_t need = saved ? p.fwd_scratch : p.infer_scratch;
   if (need > 0 && scratch == nullptr) return GSWA_ERR_NULL;
   if (misaligned(x) || misaligned(w_qkv) || misaligned(b_qkv) || misaligned(w_proj) || misaligned(b_proj) ||
@@ -132,6 +135,10 @@ int gswa_forward(const gswa_desc* desc, const void* x, const void* w_qkv, const 
   if (scratch_bytes < need) return GSWA_ERR_WORKSPACE;
   if (p.T == 0) return GSWA_OK;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (p.fast) {
+    void* carry = saved ? saved : static_cast<char*>(scratch) + p.fwd_scratch;
+    return fast_forward(p, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, y, carry, scratch, saved != nullptr, st);
+  }
   void* carry = saved ? saved : scratch;
   return generic_forward(p, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, y, carry, st);
 }
@@ -161,6 +168,9 @@ int gswa_backward(const gswa_desc* desc, const void* x, const void* w_qkv, const
     if (dbias_table && (rc = cuda_rc(cudaMemsetAsync(dbias_table, 0, nrel * p.nh * sizeof(float), st)))) return rc;
   }
   if (p.T == 0) return GSWA_OK;
+  if (p.fast)
+    return fast_backward(p, x, w_qkv, w_proj, bias_table, saved, dy, dx, dw_qkv, db_qkv, dw_proj, db_proj, dbias_table,
+                         scratch, st);
   return generic_backward(p, x, w_qkv, w_proj, bias_table, saved, dy, dx, dw_qkv, db_qkv, dw_proj, db_proj,
                           dbias_table, scratch, st);
 }
@@ -230,6 +240,20 @@ int gswa_step_host(const gswa_desc* desc, const void* x, const void* w_qkv, cons
   return cuda_rc(cudaStreamSynchronize(st));
 }
 
+int gswa_scratch_status(const gswa_desc* desc, const void* scratch, void* cuda_stream) {
+  Plan p;
+  const int rc = make_plan(desc, &p);
+  if (rc) return rc;
+  if (!p.fast || p.T == 0) return GSWA_OK;
+  if (scratch == nullptr) return GSWA_ERR_NULL;
+  int word = 0;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  int rc2 = cuda_rc(cudaMemcpyAsync(&word, scratch, sizeof(int), cudaMemcpyDeviceToHost, st));
+  if (rc2 == GSWA_OK) rc2 = cuda_rc(cudaStreamSynchronize(st));
+  if (rc2) return rc2;
+  return word == 0 ? GSWA_OK : GSWA_ERR_DEVICE;
+}
+
 int gswa_profile_enable(int on) {
   std::lock_guard<std::mutex> lk(g_prof_mu);
   g_prof_on = on != 0;
@@ -269,6 +293,7 @@ const char* gswa_status_string(int status) {
     case GSWA_ERR_UNSUPPORTED: return "layer description not supported";
     case GSWA_ERR_WORKSPACE: return "scratch or arena buffer too small";
     case GSWA_ERR_CUDA: return g_cuda_msg;
+    case GSWA_ERR_DEVICE: return "a kernel gave up waiting on an internal barrier; results are invalid";
     default: return "unknown status";
   }
 }

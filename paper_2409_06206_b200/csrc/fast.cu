@@ -1,0 +1,326 @@
+// Planner and launch sequence of the bf16 tensor-core path.
+//
+//   forward : prep_weights -> qkv_gemm (gw) -> attn_fwd -> proj_gemm (gt)
+//   backward: prep_weights -> dattn_gemm (gw: dO tiles = dy W^P per head group) -> dwproj_gemm (gr)
+//             -> attn_bwd -> dx_gemm (gt) -> dwqkv_gemm (gr)
+#include <cstring>
+
+#include "fast.cuh"
+
+namespace gswa {
+namespace {
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+constexpr size_t kSmemBudget = 215 * 1024;
+
+struct Unit {
+  int g, h0, nheads;
+};
+
+struct TokenSplit {
+  int nsplit, NB, nstages, natoms;
+};
+
+// Largest number of heads per work unit such that the QKV weight image, two activation stages and
+// the accumulators fit one SM.
+int heads_per_unit(int Cp, int dp) {
+  int best = 0;
+  for (int n = 1; n <= 3; ++n) {
+    const size_t NT = (size_t)n * 3 * dp;
+    const size_t smem = 1024 + NT * Cp * 2 + (size_t)2 * 128 * Cp * 2 + NT * 4 + 64;
+    if (smem <= kSmemBudget + 8 * 1024 && NT <= 512) best = n;
+  }
+  return best;
+}
+
+int make_units(const Plan& p, Unit* units) {
+  const int hpu = heads_per_unit(p.Cp, p.dp);
+  if (hpu == 0) return -1;
+  int n = 0;
+  for (int g = 0; g < p.G; ++g)
+    for (int h = 0; h < p.gh[g]; h += hpu) {
+      if (n == kMaxUnits) return -1;
+      units[n++] = Unit{g, p.gh0[g] + h, p.gh[g] - h < hpu ? p.gh[g] - h : hpu};
+    }
+  return n;
+}
+
+// Split of the output columns of a token GEMM with K = kvalid so that the resident weight image,
+// the staging tile and at least three ring stages fit.
+bool token_split(int C, int kvalid, TokenSplit* ts) {
+  const int natoms = (kvalid + 63) / 64;
+  for (int nsplit = 1; nsplit <= kMaxUnits; nsplit *= 2) {
+    const int NB = (int)align_up((size_t)(C + nsplit - 1) / nsplit, 32);
+    if (NB > 256) continue;
+    const size_t fixed = 1024 + (size_t)natoms * NB * 128 + (size_t)128 * NB * 2 + NB * 4 + 64;
+    if (fixed + 3 * 16384 > kSmemBudget) continue;
+    int S = (int)((kSmemBudget - fixed) / 16384);
+    if (S > 8) S = 8;
+    *ts = TokenSplit{(C + NB - 1) / NB, NB, S, natoms};
+    return true;
+  }
+  return false;
+}
+
+FastGeom make_geom(const Plan& p) {
+  FastGeom g{};
+  g.B = p.B; g.H = p.H; g.W = p.W; g.C = p.C; g.nh = p.nh; g.d = p.d; g.dp = p.dp; g.G = p.G;
+  g.nW = p.nW; g.nWw = p.nWw; g.nWh = p.nWh; g.T = p.T; g.n_windows = (long long)p.B * p.nW;
+  long long qo = 0, dO = 0, lo = 0;
+  for (int i = 0; i < p.G; ++i) {
+    g.gh[i] = p.gh[i]; g.gs[i] = p.gs[i]; g.gh0[i] = p.gh0[i];
+    g.qkv_off[i] = qo; g.do_off[i] = dO; g.l_off[i] = lo;
+    qo += g.n_windows * p.gh[i] * 3 * 64 * p.dp;
+    dO += g.n_windows * p.gh[i] * 64 * p.dp;
+    lo += g.n_windows * p.gh[i] * 64;
+  }
+  return g;
+}
+
+// Scratch layouts (byte offsets).  The first 256 bytes of either scratch hold the device error word.
+struct FwdScratch {
+  size_t img[kMaxUnits], bias[kMaxUnits], pimg[kMaxUnits], pbias[kMaxUnits], total;
+};
+struct BwdScratch {
+  size_t dO, dqkv, img[kMaxUnits], ximg[kMaxUnits], dummy, total;
+};
+
+FwdScratch fwd_layout(const Plan& p, const Unit* units, int nu, const TokenSplit& ts) {
+  FwdScratch s{};
+  size_t off = 256;
+  for (int i = 0; i < nu; ++i) {
+    const size_t NT = (size_t)units[i].nheads * 3 * p.dp;
+    s.img[i] = off; off += align_up(NT * p.Cp * 2, 256);
+    s.bias[i] = off; off += align_up(NT * 4, 256);
+  }
+  for (int i = 0; i < ts.nsplit; ++i) {
+    s.pimg[i] = off; off += align_up((size_t)ts.natoms * ts.NB * 128, 256);
+    s.pbias[i] = off; off += align_up((size_t)ts.NB * 4, 256);
+  }
+  s.total = off;
+  return s;
+}
+
+BwdScratch bwd_layout(const Plan& p, const Unit* units, int nu, const TokenSplit& tx) {
+  BwdScratch s{};
+  size_t off = 256;
+  s.dO = off; off += align_up((size_t)p.T * p.nh * p.dp * 2, 256);
+  s.dqkv = off; off += align_up((size_t)p.T * 3 * p.C * 2, 256);
+  for (int i = 0; i < nu; ++i) {
+    s.img[i] = off; off += align_up((size_t)units[i].nheads * p.dp * p.Cp * 2, 256);
+  }
+  for (int i = 0; i < tx.nsplit; ++i) {
+    s.ximg[i] = off; off += align_up((size_t)tx.natoms * tx.NB * 128, 256);
+  }
+  s.dummy = off; off += align_up((size_t)3 * p.C * p.C * 4, 256);
+  s.total = off;
+  return s;
+}
+
+int np_cols(int C) { return (int)align_up((size_t)C + 1, 64); }
+
+}  // namespace
+
+bool fast_path_ok(const Plan& p) {
+  if (p.dtype != GSWA_BF16 || (p.flags & GSWA_FLAG_GENERIC)) return false;
+  if (p.M != 8 || p.d > 32 || (p.d & 1) || (p.C & 3) || p.C > 252 || p.G > 4) return false;
+  if (p.T >= (1LL << 30) / 4) return false;
+  Plan q = p;
+  q.dp = p.d <= 16 ? 16 : 32;
+  q.Cp = (int)align_up((size_t)p.C, 64);
+  Unit units[kMaxUnits];
+  if (make_units(q, units) <= 0) return false;
+  TokenSplit a, b;
+  return token_split(p.C, p.C, &a) && token_split(p.C, 3 * p.C, &b);
+}
+
+void fast_plan_sizes(Plan* p) {
+  p->fast = 1;
+  p->dp = p->d <= 16 ? 16 : 32;
+  p->Cp = (int)align_up((size_t)p->C, 64);
+  Unit units[kMaxUnits];
+  const int nu = make_units(*p, units);
+  TokenSplit tp, tx;
+  token_split(p->C, p->C, &tp);
+  token_split(p->C, 3 * p->C, &tx);
+  const size_t T = (size_t)p->T;
+  p->off_qkv = 0;
+  p->off_A = align_up(T * 3 * p->nh * p->dp * 2, 256);
+  p->off_L = p->off_A + align_up(T * p->C * 2, 256);
+  p->saved_bytes = p->off_L + align_up(T * p->nh * 4, 256);
+  p->fwd_scratch = fwd_layout(*p, units, nu, tp).total;
+  p->infer_scratch = p->fwd_scratch + p->saved_bytes;
+  p->bwd_scratch = bwd_layout(*p, units, nu, tx).total;
+}
+
+static void attn_units(const Plan& p, const FastGeom& geo, const Unit* units, int nu, AttnLaunch* L) {
+  L->geo = geo;
+  L->nunits = nu;
+  for (int i = 0; i < nu; ++i) {
+    const Unit& u = units[i];
+    const int hl0 = u.h0 - p.gh0[u.g], gh = p.gh[u.g];
+    AttnUnit& a = L->u[i];
+    a.g = u.g; a.h0 = u.h0; a.nheads = u.nheads; a.s = p.gs[u.g];
+    a.qkv_off = geo.qkv_off[u.g] + (long long)hl0 * 3 * 64 * p.dp;
+    a.do_off = geo.do_off[u.g] + (long long)hl0 * 64 * p.dp;
+    a.l_off = geo.l_off[u.g] + (long long)hl0 * 64;
+    a.qkv_wstride = (long long)gh * 3 * 64 * p.dp;
+    a.do_wstride = (long long)gh * 64 * p.dp;
+    a.l_wstride = (long long)gh * 64;
+  }
+}
+
+int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
+                 const void* b_proj, const void* table, void* y, void* saved, void* scratch, bool want_L,
+                 cudaStream_t st) {
+  using bf = __nv_bfloat16;
+  Unit units[kMaxUnits];
+  const int nu = make_units(p, units);
+  TokenSplit tp;
+  if (nu <= 0 || !token_split(p.C, p.C, &tp)) return GSWA_ERR_UNSUPPORTED;
+  const FwdScratch fs = fwd_layout(p, units, nu, tp);
+  const FastGeom geo = make_geom(p);
+  char* sc = static_cast<char*>(scratch);
+  char* sv = static_cast<char*>(saved);
+  int* err = reinterpret_cast<int*>(sc);
+  bf* qkv = reinterpret_cast<bf*>(sv + p.off_qkv);
+  bf* A = reinterpret_cast<bf*>(sv + p.off_A);
+  float* Lt = reinterpret_cast<float*>(sv + p.off_L);
+  if (cudaMemsetAsync(err, 0, 256, st) != cudaSuccess) return check_launch();
+
+  PrepJob jobs[16];
+  int nj = 0;
+  for (int i = 0; i < nu; ++i)
+    jobs[nj++] = PrepJob{PREP_QKV, (const bf*)w_qkv, (const bf*)b_qkv, (unsigned char*)sc + fs.img[i],
+                         (float*)(sc + fs.bias[i]), p.C, p.d, p.dp, units[i].h0, units[i].nheads, 0,
+                         units[i].nheads * 3 * p.dp, p.Cp};
+  for (int i = 0; i < tp.nsplit; ++i)
+    jobs[nj++] = PrepJob{PREP_PROJ, (const bf*)w_proj, (const bf*)b_proj, (unsigned char*)sc + fs.pimg[i],
+                         (float*)(sc + fs.pbias[i]), p.C, p.d, p.dp, 0, 0, i * tp.NB, tp.NB, tp.natoms * 64};
+  int rc = launch_prep(jobs, nj, st);
+  if (rc) return rc;
+
+  GWLaunch gw{};
+  gw.err = err;
+  for (int i = 0; i < nu; ++i) {
+    const Unit& u = units[i];
+    GWUnit& w = gw.u[i];
+    w.A = (const bf*)x; w.lda = p.C; w.kvalid = p.C;
+    w.H = p.H; w.W = p.W; w.s = p.gs[u.g]; w.nW = p.nW; w.nWw = p.nWw; w.n_windows = geo.n_windows;
+    w.Bimg = (const unsigned char*)sc + fs.img[i];
+    w.bias = (const float*)(sc + fs.bias[i]);
+    w.out = qkv + geo.qkv_off[u.g] + (long long)(u.h0 - p.gh0[u.g]) * 3 * 64 * p.dp;
+    w.win_stride = (long long)p.gh[u.g] * 3 * 64 * p.dp;
+    w.nchunks = u.nheads; w.cw = 3 * p.dp; w.q_every3 = 1;
+    w.qscale = 1.0f / sqrtf((float)p.d);
+  }
+  if ((rc = launch_gw(gw, nu, p.Cp, p.dp, st, "qkv_gemm"))) return rc;
+
+  AttnLaunch al{};
+  attn_units(p, geo, units, nu, &al);
+  al.qkv = qkv; al.table = (const bf*)table; al.A = A; al.Lt = want_L ? Lt : nullptr;
+  al.scale = 1.0f / sqrtf((float)p.d);
+  if ((rc = launch_attn_fwd(al, st))) return rc;
+
+  GTLaunch gt{};
+  gt.A = A; gt.lda = p.C; gt.kvalid = p.C; gt.natoms = tp.natoms; gt.rows = p.T;
+  gt.out = (bf*)y; gt.ldo = p.C; gt.NB = tp.NB; gt.nstages = tp.nstages; gt.err = err;
+  for (int i = 0; i < tp.nsplit; ++i) {
+    const int col0 = i * tp.NB;
+    gt.s[i] = GTSplit{(const unsigned char*)sc + fs.pimg[i], (const float*)(sc + fs.pbias[i]), col0,
+                      (p.C - col0 < tp.NB ? p.C - col0 : tp.NB)};
+  }
+  return launch_gt(gt, tp.nsplit, st, "proj_gemm");
+}
+
+int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w_proj, const void* table,
+                  const void* saved, const void* dy, void* dx, float* dw_qkv, float* db_qkv, float* dw_proj,
+                  float* db_proj, float* dtable, void* scratch, cudaStream_t st) {
+  using bf = __nv_bfloat16;
+  Unit units[kMaxUnits];
+  const int nu = make_units(p, units);
+  TokenSplit tx;
+  if (nu <= 0 || !token_split(p.C, 3 * p.C, &tx)) return GSWA_ERR_UNSUPPORTED;
+  const BwdScratch bs = bwd_layout(p, units, nu, tx);
+  const FastGeom geo = make_geom(p);
+  char* sc = static_cast<char*>(scratch);
+  const char* sv = static_cast<const char*>(saved);
+  int* err = reinterpret_cast<int*>(sc);
+  const bf* qkv = reinterpret_cast<const bf*>(sv + p.off_qkv);
+  const bf* A = reinterpret_cast<const bf*>(sv + p.off_A);
+  const float* Lt = reinterpret_cast<const float*>(sv + p.off_L);
+  bf* dO = reinterpret_cast<bf*>(sc + bs.dO);
+  bf* dqkv = reinterpret_cast<bf*>(sc + bs.dqkv);
+  float* dummy = reinterpret_cast<float*>(sc + bs.dummy);
+  if (cudaMemsetAsync(err, 0, 256, st) != cudaSuccess) return check_launch();
+
+  PrepJob jobs[16];
+  int nj = 0;
+  for (int i = 0; i < nu; ++i)
+    jobs[nj++] = PrepJob{PREP_PROJ_T, (const bf*)w_proj, nullptr, (unsigned char*)sc + bs.img[i], nullptr, p.C, p.d,
+                         p.dp, units[i].h0, units[i].nheads, 0, units[i].nheads * p.dp, p.Cp};
+  for (int i = 0; i < tx.nsplit; ++i)
+    jobs[nj++] = PrepJob{PREP_QKV_T, (const bf*)w_qkv, nullptr, (unsigned char*)sc + bs.ximg[i], nullptr, p.C, p.d,
+                         p.dp, 0, 0, i * tx.NB, tx.NB, tx.natoms * 64};
+  int rc = launch_prep(jobs, nj, st);
+  if (rc) return rc;
+
+  // dO tiles = dy W^P restricted to each unit's heads, rows gathered in that group's window order
+  GWLaunch gw{};
+  gw.err = err;
+  for (int i = 0; i < nu; ++i) {
+    const Unit& u = units[i];
+    GWUnit& w = gw.u[i];
+    w.A = (const bf*)dy; w.lda = p.C; w.kvalid = p.C;
+    w.H = p.H; w.W = p.W; w.s = p.gs[u.g]; w.nW = p.nW; w.nWw = p.nWw; w.n_windows = geo.n_windows;
+    w.Bimg = (const unsigned char*)sc + bs.img[i];
+    w.bias = nullptr;
+    w.out = dO + geo.do_off[u.g] + (long long)(u.h0 - p.gh0[u.g]) * 64 * p.dp;
+    w.win_stride = (long long)p.gh[u.g] * 64 * p.dp;
+    w.nchunks = 1; w.cw = u.nheads * p.dp; w.q_every3 = 0; w.qscale = 1.f;
+  }
+  if ((rc = launch_gw(gw, nu, p.Cp, p.dp, st, "dattn_gemm"))) return rc;
+
+  const int sms = 148;
+  if (dw_proj || db_proj) {
+    GRLaunch gr{};
+    gr.L = (const bf*)dy; gr.ldl = p.C; gr.mvalid = p.C;
+    gr.R = A; gr.ldr = p.C; gr.nvalid = p.C; gr.rows = p.T; gr.NP = np_cols(p.C);
+    const int mblocks = (p.C + 127) / 128;
+    long long ns = sms / mblocks, cap = (p.T + 63) / 64;
+    gr.nsplit = (int)(ns < cap ? (ns < 1 ? 1 : ns) : cap);
+    gr.out = dw_proj ? dw_proj : dummy; gr.colsum = db_proj; gr.err = err;
+    if ((rc = launch_gr(gr, st, "dwproj_gemm"))) return rc;
+  }
+
+  AttnLaunch al{};
+  attn_units(p, geo, units, nu, &al);
+  al.qkv = qkv; al.table = (const bf*)table; al.Lt = const_cast<float*>(Lt); al.dO = dO; al.dqkv = dqkv;
+  al.dtable = dtable; al.scale = 1.0f / sqrtf((float)p.d);
+  if ((rc = launch_attn_bwd(al, st))) return rc;
+
+  if (dx) {
+    GTLaunch gt{};
+    gt.A = dqkv; gt.lda = 3 * p.C; gt.kvalid = 3 * p.C; gt.natoms = tx.natoms; gt.rows = p.T;
+    gt.out = (bf*)dx; gt.ldo = p.C; gt.NB = tx.NB; gt.nstages = tx.nstages; gt.err = err;
+    for (int i = 0; i < tx.nsplit; ++i) {
+      const int col0 = i * tx.NB;
+      gt.s[i] = GTSplit{(const unsigned char*)sc + bs.ximg[i], nullptr, col0, (p.C - col0 < tx.NB ? p.C - col0 : tx.NB)};
+    }
+    if ((rc = launch_gt(gt, tx.nsplit, st, "dx_gemm"))) return rc;
+  }
+  if (dw_qkv || db_qkv) {
+    GRLaunch gr{};
+    gr.L = dqkv; gr.ldl = 3 * p.C; gr.mvalid = 3 * p.C;
+    gr.R = (const bf*)x; gr.ldr = p.C; gr.nvalid = p.C; gr.rows = p.T; gr.NP = np_cols(p.C);
+    const int mblocks = (3 * p.C + 127) / 128;
+    long long ns = sms / mblocks, cap = (p.T + 63) / 64;
+    gr.nsplit = (int)(ns < cap ? (ns < 1 ? 1 : ns) : cap);
+    gr.out = dw_qkv ? dw_qkv : dummy; gr.colsum = db_qkv; gr.err = err;
+    if ((rc = launch_gr(gr, st, "dwqkv_gemm"))) return rc;
+  }
+  return GSWA_OK;
+}
+
+}  // namespace gswa

@@ -1,0 +1,130 @@
+// Data layout of the bf16 tensor-core path (window 8x8, head dim <= 32) and the launch interfaces
+// of its kernels.
+//
+// "Tiled" buffers hold one contiguous block per (group, window, head, kind): [64 slots][DP] bf16 with
+// the head dim padded to DP (16 or 32).  Windows of one group are numbered b*nW + w.  The QKV
+// projection writes q,k,v straight into this layout (cyclic shift + window partition happen in its
+// epilogue addressing), so the attention kernels read contiguous, 16-byte aligned tiles:
+//   qkv tiles of group g : base + qkv_off[g] + window*(gh*3*64*DP) + ((hl*3 + kind)*64 + slot)*DP + c
+//   dO  tiles of group g : base + do_off[g]  + window*(gh*64*DP)   + (hl*64 + slot)*DP + c
+//   L   tiles of group g : base + l_off[g]   + window*(gh*64)      +  hl*64 + slot            (float)
+// "Token-major" buffers are packed [T, cols] rows in original token order (attention output A[T,C],
+// dqkv[T,3C]); the attention epilogues undo partition and shift when they store into them.
+#pragma once
+
+#include "gswa_internal.h"
+
+namespace gswa {
+
+constexpr int kMaxUnits = 8;   // (group, head range) work units per launch
+
+struct FastGeom {
+  int B, H, W, C, nh, d, dp, G;
+  int nW, nWw, nWh;
+  long long T, n_windows;          // n_windows = B*nW
+  int gh[kMaxGroups], gs[kMaxGroups], gh0[kMaxGroups];
+  long long qkv_off[kMaxGroups], do_off[kMaxGroups], l_off[kMaxGroups];   // element offsets
+};
+
+// ---- window GEMM: rows gathered in window order from a packed [T, lda] source, output to tiles
+struct GWUnit {
+  const __nv_bfloat16* A;      // source rows (x or dy), pitch lda elements, `kvalid` valid columns
+  int lda, kvalid;
+  int H, W, s, nW, nWw;
+  long long n_windows;
+  const unsigned char* Bimg;   // weight image: [KP/64 atoms][NT rows][128 B], rows swizzled
+  const float* bias;           // [NT] or nullptr
+  __nv_bfloat16* out;          // tile base of this unit (already offset to its first block)
+  long long win_stride;        // elements between consecutive windows
+  int nchunks, cw;             // NT = nchunks*cw accumulator columns; cw multiple of 16 and of DP
+  int q_every3;                // 1: blocks with index % 3 == 0 are scaled by qscale
+  float qscale;
+};
+struct GWLaunch {
+  GWUnit u[kMaxUnits];
+  int* err;
+};
+
+// ---- token GEMM: rows in token order from packed [T, lda], output packed rows [T, ldo]
+struct GTSplit {
+  const unsigned char* Bimg;   // [KP/64 atoms][NB rows][128 B]
+  const float* bias;           // [NB] or nullptr
+  int col0, ncols;             // output columns [col0, col0+ncols) of each row
+};
+struct GTLaunch {
+  const __nv_bfloat16* A;
+  int lda, kvalid, natoms;     // natoms = KP/64
+  long long rows;
+  __nv_bfloat16* out;
+  int ldo;
+  int NB;                      // accumulator columns per CTA (multiple of 32, <= 256)
+  int nstages;
+  GTSplit s[kMaxUnits];
+  int* err;
+};
+
+// ---- reduction GEMM: out[m, n] += sum_t L[t, m] R[t, n], plus column sums of L via a ones column
+struct GRLaunch {
+  const __nv_bfloat16* L;      // [rows, ldl], mvalid valid columns
+  int ldl, mvalid;
+  const __nv_bfloat16* R;      // [rows, ldr], nvalid valid columns
+  int ldr, nvalid;
+  long long rows;
+  int NP;                      // padded N (multiple of 64, > nvalid so that column nvalid can carry ones)
+  int nsplit;                  // token splits
+  float* out;                  // [mvalid, nvalid] float, accumulated with atomics
+  float* colsum;               // [mvalid] or nullptr: sum_t L[t, m]
+  int* err;
+};
+
+int launch_gw(const GWLaunch& L, int nunits, int Cp, int dp, cudaStream_t st, const char* name);
+int launch_gt(const GTLaunch& L, int nsplits, cudaStream_t st, const char* name);
+int launch_gr(const GRLaunch& L, cudaStream_t st, const char* name);
+
+// Weight images (shared-memory images of the B operands, built once per call by a small kernel).
+enum PrepMode { PREP_QKV = 0, PREP_PROJ_T = 1, PREP_PROJ = 2, PREP_QKV_T = 3 };
+struct PrepJob {
+  int mode;
+  const __nv_bfloat16* W;      // source weight
+  const __nv_bfloat16* b;      // source bias or nullptr
+  unsigned char* img;
+  float* bias_out;             // or nullptr
+  int C, d, dp, h0, nheads;    // head range for the per-head modes
+  int n0, NT, KP;              // first output row (PREP_PROJ / PREP_QKV_T), rows, padded K
+};
+int launch_prep(const PrepJob* jobs, int njobs, cudaStream_t st);
+
+// ---- attention (mma.sync m16n8k16, softmax in registers)
+struct AttnUnit {
+  int g, h0, nheads;           // group, first head (global index), heads in this unit
+  int s;
+  long long qkv_off, do_off, l_off;      // element offsets of the unit's first block inside window 0
+  long long qkv_wstride, do_wstride, l_wstride;
+};
+struct AttnLaunch {
+  FastGeom geo;
+  AttnUnit u[kMaxUnits];
+  int nunits;
+  const __nv_bfloat16* qkv;    // tile base
+  const __nv_bfloat16* table;  // [(2M-1)^2, nh]
+  __nv_bfloat16* A;            // fwd: [T, C] out
+  float* Lt;                   // L tiles (fwd: out or nullptr; bwd: in)
+  const __nv_bfloat16* dO;     // bwd: dO tiles
+  __nv_bfloat16* dqkv;         // bwd: [T, 3C] out
+  float* dtable;               // bwd: [(2M-1)^2, nh] float, atomics; or nullptr
+  float scale;
+};
+int launch_attn_fwd(const AttnLaunch& L, cudaStream_t st);
+int launch_attn_bwd(const AttnLaunch& L, cudaStream_t st);
+
+// ---- orchestration
+bool fast_path_ok(const Plan& p);
+void fast_plan_sizes(Plan* p);
+int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
+                 const void* b_proj, const void* table, void* y, void* saved, void* scratch, bool want_L,
+                 cudaStream_t st);
+int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w_proj, const void* table,
+                  const void* saved, const void* dy, void* dx, float* dw_qkv, float* db_qkv, float* dw_proj,
+                  float* db_proj, float* dtable, void* scratch, cudaStream_t st);
+
+}  // namespace gswa

@@ -1,0 +1,449 @@
+// Window attention of the bf16 path, forward and recompute-based backward (Eq. 6 `Attn`, with the
+// relative-position bias and the shifted-window mask).  One 8x8 window is a 64 x 64 x d problem per
+// head: far too small to feed a 128-row tcgen05 tile without packing unrelated windows, and its cost
+// is dominated by the softmax and the index work, so these kernels use warp-level mma.sync
+// m16n8k16 with the score tile, the softmax and the probability operand all kept in registers
+// (row statistics by quad shuffles).  q, k, v arrive as contiguous per-(window, head) tiles; the
+// mask is evaluated from per-slot region labels (never a [windows, 64, 64] tensor) and only in the
+// windows of the last row / column of a shifted group; window reverse and reverse shift are the
+// address arithmetic of the output stores.
+//
+// The backward pass keeps only the row log-sum-exp from the forward pass: P = exp(S - L) is rebuilt
+// per window, D = rowsum(P * dP) replaces the usual dO.O term, and P / dS cross from the
+// query-major phase (dQ) to the key-major phase (dK, dV) through shared memory.
+#include "fast.cuh"
+#include "gswa_index.cuh"
+
+namespace gswa {
+namespace {
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+__device__ __forceinline__ void ldsm_x4(uint32_t* r, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t* r, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void mma16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
+
+// Shared-memory image of a [64][DP] tile: 16-byte chunks of a row permuted so that ldmatrix of
+// eight consecutive rows is bank-conflict free.
+template <int DP>
+__device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
+  constexpr int CH = DP / 8;                // chunks per row (4 or 2)
+  return (uint32_t)(row * (DP * 2) + ((chunk ^ ((row / (8 / CH)) % CH)) << 4));
+}
+// [64][64] bf16 matrices (P, dS): 128-byte rows, chunk ^= row & 7.
+__device__ __forceinline__ uint32_t sq_off(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
+
+template <int DP>
+__device__ __forceinline__ void load_tiles(unsigned char* dst, const __nv_bfloat16* src, int nblocks, int tid, int nt) {
+  constexpr int CH = DP / 8;
+  const int nchunks = nblocks * 64 * CH;
+  const uint32_t d0 = smem_u32(dst);
+  for (int ci = tid; ci < nchunks; ci += nt) {
+    const int rowg = ci / CH, chunk = ci % CH;
+    cp_async16(d0 + (rowg >> 6) * (64 * DP * 2) + tile_off<DP>(rowg & 63, chunk),
+               reinterpret_cast<const unsigned char*>(src) + (size_t)ci * 16);
+  }
+}
+
+// S (16 rows x 64 keys) = Q K^T for the warp's rows; returns accumulators in s[8][4].
+template <int DP>
+__device__ __forceinline__ void qk_scores(float (*s)[4], uint32_t q_base, uint32_t k_base, int r0, int lane) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+#pragma unroll
+  for (int kk = 0; kk < DP / 16; ++kk) {
+    uint32_t a[4];
+    ldsm_x4(a, q_base + tile_off<DP>(r0 + (lane & 15), 2 * kk + (lane >> 4)));
+#pragma unroll
+    for (int jp = 0; jp < 4; ++jp) {
+      uint32_t b[4];
+      ldsm_x4(b, k_base + tile_off<DP>(16 * jp + (lane & 7) + ((lane >> 4) << 3), 2 * kk + ((lane >> 3) & 1)));
+      mma16816(s[2 * jp], a, b[0], b[1]);
+      mma16816(s[2 * jp + 1], a, b[2], b[3]);
+    }
+  }
+}
+
+// acc (16 x DP) += A(16 x 64, from packed register fragments of `pf`) * B(64 x DP) with B read
+// transposed from a [64][DP] tile (rows = contraction index).
+template <int DP>
+__device__ __forceinline__ void regs_times_tile(float (*acc)[4], const float (*pf)[4], uint32_t b_base, int lane) {
+#pragma unroll
+  for (int kk = 0; kk < 4; ++kk) {
+    uint32_t a[4];
+    a[0] = pack2(pf[2 * kk][0], pf[2 * kk][1]);
+    a[1] = pack2(pf[2 * kk][2], pf[2 * kk][3]);
+    a[2] = pack2(pf[2 * kk + 1][0], pf[2 * kk + 1][1]);
+    a[3] = pack2(pf[2 * kk + 1][2], pf[2 * kk + 1][3]);
+#pragma unroll
+    for (int jn = 0; jn < DP / 16; ++jn) {
+      uint32_t b[4];
+      ldsm_x4_t(b, b_base + tile_off<DP>(16 * kk + (lane & 7) + (((lane >> 3) & 1) << 3), 2 * jn + (lane >> 4)));
+      mma16816(acc[2 * jn], a, b[0], b[1]);
+      mma16816(acc[2 * jn + 1], a, b[2], b[3]);
+    }
+  }
+}
+
+struct WinCtx {
+  int b, wi, wj;
+  bool masked;
+};
+
+__device__ __forceinline__ WinCtx window_setup(const FastGeom& g, int s, long long win, int* tok, unsigned char* reg,
+                                               int tid) {
+  WinCtx c;
+  c.b = (int)(win / g.nW);
+  const int w = (int)(win % g.nW);
+  c.wi = w / g.nWw;
+  c.wj = w % g.nWw;
+  c.masked = s > 0 && (c.wi == g.nWh - 1 || c.wj == g.nWw - 1);
+  if (tid < 64) {
+    int i, j, r;
+    slot_to_token(g.H, g.W, 8, s, w, tid, &i, &j, &r);
+    tok[tid] = (c.b * g.H + i) * g.W + j;
+    reg[tid] = (unsigned char)r;
+  }
+  return c;
+}
+
+// Adds the relative-position bias, applies the mask and moves the scores to the log2 domain.
+__device__ __forceinline__ void bias_and_mask(float (*s)[4], const float* tab, const unsigned char* reg, bool masked,
+                                              int p0, int t) {
+  const int pa0 = p0 >> 3, pc0 = p0 & 7;   // rows p0 and p0 + 8: same column in the window, next row
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int pa = pa0 + (e >> 1), qc = 2 * t + (e & 1);
+      const int rel = (pa - j + 7) * 15 + (pc0 - qc + 7);
+      s[j][e] = (s[j][e] + tab[rel]) * kLog2e;
+    }
+  }
+  if (masked) {
+    const unsigned char r0 = reg[p0], r1 = reg[p0 + 8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const unsigned char q0 = reg[8 * j + 2 * t], q1 = reg[8 * j + 2 * t + 1];
+      if (q0 != r0) s[j][0] = -INFINITY;
+      if (q1 != r0) s[j][1] = -INFINITY;
+      if (q0 != r1) s[j][2] = -INFINITY;
+      if (q1 != r1) s[j][3] = -INFINITY;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// forward: one CTA per (window, unit); 4 warps per head, 16 query rows per warp
+// ------------------------------------------------------------------------------------------
+template <int DP>
+__global__ void __launch_bounds__(512) attn_fwd_kernel(const __grid_constant__ AttnLaunch L) {
+  const AttnUnit& u = L.u[blockIdx.y];
+  const FastGeom& g = L.geo;
+  extern __shared__ __align__(128) unsigned char sm[];
+  const int nh_u = u.nheads;
+  unsigned char* tiles = sm;
+  float* tab = reinterpret_cast<float*>(tiles + (size_t)nh_u * 3 * 64 * DP * 2);
+  int* tok = reinterpret_cast<int*>(tab + nh_u * 225);
+  unsigned char* reg = reinterpret_cast<unsigned char*>(tok + 64);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int nt = nh_u * 128;
+  if (tid >= nt) return;
+  const long long win = blockIdx.x;
+
+  load_tiles<DP>(tiles, L.qkv + u.qkv_off + win * u.qkv_wstride, nh_u * 3, tid, nt);
+  for (int e = tid; e < nh_u * 225; e += nt)
+    tab[e] = __bfloat162float(L.table[(e % 225) * g.nh + u.h0 + e / 225]);
+  const WinCtx wc = window_setup(g, u.s, win, tok, reg, tid);
+  cp_async_wait_all();
+  __syncthreads();
+
+  const int hl = warp >> 2, r0 = (warp & 3) * 16, gq = lane >> 2, t = lane & 3;
+  const uint32_t q_base = smem_u32(tiles + (size_t)(hl * 3 + 0) * 64 * DP * 2);
+  const uint32_t k_base = q_base + 64 * DP * 2, v_base = k_base + 64 * DP * 2;
+  float s[8][4];
+  qk_scores<DP>(s, q_base, k_base, r0, lane);
+  const int p0 = r0 + gq;
+  bias_and_mask(s, tab + hl * 225, reg, wc.masked, p0, t);
+
+  float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    m0 = fmaxf(m0, fmaxf(s[j][0], s[j][1]));
+    m1 = fmaxf(m1, fmaxf(s[j][2], s[j][3]));
+  }
+  m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1));
+  m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
+  m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1));
+  m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
+  float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    s[j][0] = exp2f(s[j][0] - m0);
+    s[j][1] = exp2f(s[j][1] - m0);
+    s[j][2] = exp2f(s[j][2] - m1);
+    s[j][3] = exp2f(s[j][3] - m1);
+    sum0 += s[j][0] + s[j][1];
+    sum1 += s[j][2] + s[j][3];
+  }
+  sum0 += __shfl_xor_sync(0xffffffffu, sum0, 1);
+  sum0 += __shfl_xor_sync(0xffffffffu, sum0, 2);
+  sum1 += __shfl_xor_sync(0xffffffffu, sum1, 1);
+  sum1 += __shfl_xor_sync(0xffffffffu, sum1, 2);
+
+  float o[DP / 8][4];
+#pragma unroll
+  for (int j = 0; j < DP / 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
+  regs_times_tile<DP>(o, s, v_base, lane);
+
+  const float inv0 = 1.f / sum0, inv1 = 1.f / sum1;
+  const int h = u.h0 + hl;
+  __nv_bfloat16* out0 = L.A + (long long)tok[p0] * g.C + h * g.d;
+  __nv_bfloat16* out1 = L.A + (long long)tok[p0 + 8] * g.C + h * g.d;
+#pragma unroll
+  for (int jn = 0; jn < DP / 8; ++jn) {
+    const int col = 8 * jn + 2 * t;
+    if (col < g.d) {
+      *reinterpret_cast<uint32_t*>(out0 + col) = pack2(o[jn][0] * inv0, o[jn][1] * inv0);
+      *reinterpret_cast<uint32_t*>(out1 + col) = pack2(o[jn][2] * inv1, o[jn][3] * inv1);
+    }
+  }
+  if (L.Lt != nullptr && t == 0) {
+    float* lt = L.Lt + u.l_off + win * u.l_wstride + hl * 64;
+    lt[p0] = m0 * kLn2 + logf(sum0);
+    lt[p0 + 8] = m1 * kLn2 + logf(sum1);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// backward: persistent CTAs stride over the windows of a unit
+// ------------------------------------------------------------------------------------------
+template <int DP>
+__global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant__ AttnLaunch L) {
+  const AttnUnit& u = L.u[blockIdx.y];
+  const FastGeom& g = L.geo;
+  extern __shared__ __align__(128) unsigned char sm[];
+  const int nh_u = u.nheads;
+  constexpr int kTile = 64 * DP * 2;
+  unsigned char* tiles = sm;                                   // q,k,v per head
+  unsigned char* dot = tiles + (size_t)nh_u * 3 * kTile;       // dO per head
+  unsigned char* Ps = dot + (size_t)nh_u * kTile;              // [head][64][64] bf16
+  unsigned char* dSs = Ps + (size_t)nh_u * 8192;
+  float* tab = reinterpret_cast<float*>(dSs + (size_t)nh_u * 8192);
+  float* hist = tab + nh_u * 225;
+  float* Lrow = hist + nh_u * 225;
+  int* tok = reinterpret_cast<int*>(Lrow + nh_u * 64);
+  unsigned char* reg = reinterpret_cast<unsigned char*>(tok + 64);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int nt = nh_u * 128;
+  if (tid >= nt) return;
+
+  for (int e = tid; e < nh_u * 225; e += nt) {
+    tab[e] = __bfloat162float(L.table[(e % 225) * g.nh + u.h0 + e / 225]);
+    hist[e] = 0.f;
+  }
+  const int hl = warp >> 2, r0 = (warp & 3) * 16, gq = lane >> 2, t = lane & 3;
+  const int h = u.h0 + hl;
+  const uint32_t q_base = smem_u32(tiles + (size_t)(hl * 3) * kTile);
+  const uint32_t k_base = q_base + kTile, v_base = k_base + kTile;
+  const uint32_t do_base = smem_u32(dot + (size_t)hl * kTile);
+  unsigned char* Ph = Ps + (size_t)hl * 8192;
+  unsigned char* dSh = dSs + (size_t)hl * 8192;
+  const int p0 = r0 + gq;
+  float dsum[8][4];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) dsum[j][0] = dsum[j][1] = dsum[j][2] = dsum[j][3] = 0.f;
+
+  for (long long win = blockIdx.x; win < g.n_windows; win += gridDim.x) {
+    __syncthreads();   // previous window's tiles, P and dS are no longer read
+    load_tiles<DP>(tiles, L.qkv + u.qkv_off + win * u.qkv_wstride, nh_u * 3, tid, nt);
+    load_tiles<DP>(dot, L.dO + u.do_off + win * u.do_wstride, nh_u, tid, nt);
+    for (int e = tid; e < nh_u * 64; e += nt) Lrow[e] = L.Lt[u.l_off + win * u.l_wstride + e];
+    const WinCtx wc = window_setup(g, u.s, win, tok, reg, tid);
+    cp_async_wait_all();
+    __syncthreads();
+
+    // ---- query-major phase: this warp owns query rows r0 .. r0+15 of head hl
+    float s[8][4];
+    qk_scores<DP>(s, q_base, k_base, r0, lane);
+    bias_and_mask(s, tab + hl * 225, reg, wc.masked, p0, t);
+    const float l0 = Lrow[hl * 64 + p0] * kLog2e, l1 = Lrow[hl * 64 + p0 + 8] * kLog2e;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      s[j][0] = exp2f(s[j][0] - l0);
+      s[j][1] = exp2f(s[j][1] - l0);
+      s[j][2] = exp2f(s[j][2] - l1);
+      s[j][3] = exp2f(s[j][3] - l1);
+    }
+    float dp[8][4];
+    qk_scores<DP>(dp, do_base, v_base, r0, lane);          // dP = dO V^T
+    float d0 = 0.f, d1 = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      d0 += s[j][0] * dp[j][0] + s[j][1] * dp[j][1];
+      d1 += s[j][2] * dp[j][2] + s[j][3] * dp[j][3];
+    }
+    d0 += __shfl_xor_sync(0xffffffffu, d0, 1);
+    d0 += __shfl_xor_sync(0xffffffffu, d0, 2);
+    d1 += __shfl_xor_sync(0xffffffffu, d1, 1);
+    d1 += __shfl_xor_sync(0xffffffffu, d1, 2);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      dp[j][0] = s[j][0] * (dp[j][0] - d0);
+      dp[j][1] = s[j][1] * (dp[j][1] - d0);
+      dp[j][2] = s[j][2] * (dp[j][2] - d1);
+      dp[j][3] = s[j][3] * (dp[j][3] - d1);
+      dsum[j][0] += dp[j][0];
+      dsum[j][1] += dp[j][1];
+      dsum[j][2] += dp[j][2];
+      dsum[j][3] += dp[j][3];
+      *reinterpret_cast<uint32_t*>(Ph + sq_off(p0, j) + t * 4) = pack2(s[j][0], s[j][1]);
+      *reinterpret_cast<uint32_t*>(Ph + sq_off(p0 + 8, j) + t * 4) = pack2(s[j][2], s[j][3]);
+      *reinterpret_cast<uint32_t*>(dSh + sq_off(p0, j) + t * 4) = pack2(dp[j][0], dp[j][1]);
+      *reinterpret_cast<uint32_t*>(dSh + sq_off(p0 + 8, j) + t * 4) = pack2(dp[j][2], dp[j][3]);
+    }
+    {
+      float dq[DP / 8][4];
+#pragma unroll
+      for (int j = 0; j < DP / 8; ++j) dq[j][0] = dq[j][1] = dq[j][2] = dq[j][3] = 0.f;
+      regs_times_tile<DP>(dq, dp, k_base, lane);             // dQ = dS K
+      __nv_bfloat16* o0 = L.dqkv + (long long)tok[p0] * 3 * g.C + h * g.d;
+      __nv_bfloat16* o1 = L.dqkv + (long long)tok[p0 + 8] * 3 * g.C + h * g.d;
+#pragma unroll
+      for (int jn = 0; jn < DP / 8; ++jn) {
+        const int col = 8 * jn + 2 * t;
+        if (col < g.d) {
+          *reinterpret_cast<uint32_t*>(o0 + col) = pack2(dq[jn][0] * L.scale, dq[jn][1] * L.scale);
+          *reinterpret_cast<uint32_t*>(o1 + col) = pack2(dq[jn][2] * L.scale, dq[jn][3] * L.scale);
+        }
+      }
+    }
+    __syncthreads();
+
+    // ---- key-major phase: this warp owns keys r0 .. r0+15: dV = P^T dO, dK = dS^T Q
+    float dv[DP / 8][4], dk[DP / 8][4];
+#pragma unroll
+    for (int j = 0; j < DP / 8; ++j)
+      dv[j][0] = dv[j][1] = dv[j][2] = dv[j][3] = dk[j][0] = dk[j][1] = dk[j][2] = dk[j][3] = 0.f;
+    const uint32_t p_addr = smem_u32(Ph), ds_addr = smem_u32(dSh);
+    const int kc = (warp & 3) * 2;   // first 16-byte key chunk of this warp
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      uint32_t ap[4], ad[4];
+      const int qrow = 16 * kk + (lane & 7) + (((lane >> 4) & 1) << 3);
+      const int chunk = kc + ((lane >> 3) & 1);
+      ldsm_x4_t(ap, p_addr + sq_off(qrow, chunk));
+      ldsm_x4_t(ad, ds_addr + sq_off(qrow, chunk));
+#pragma unroll
+      for (int jn = 0; jn < DP / 16; ++jn) {
+        uint32_t b[4];
+        const int brow = 16 * kk + (lane & 7) + (((lane >> 3) & 1) << 3);
+        ldsm_x4_t(b, do_base + tile_off<DP>(brow, 2 * jn + (lane >> 4)));
+        mma16816(dv[2 * jn], ap, b[0], b[1]);
+        mma16816(dv[2 * jn + 1], ap, b[2], b[3]);
+        ldsm_x4_t(b, q_base + tile_off<DP>(brow, 2 * jn + (lane >> 4)));
+        mma16816(dk[2 * jn], ad, b[0], b[1]);
+        mma16816(dk[2 * jn + 1], ad, b[2], b[3]);
+      }
+    }
+    {
+      __nv_bfloat16* o0 = L.dqkv + (long long)tok[p0] * 3 * g.C + g.C + h * g.d;
+      __nv_bfloat16* o1 = L.dqkv + (long long)tok[p0 + 8] * 3 * g.C + g.C + h * g.d;
+#pragma unroll
+      for (int jn = 0; jn < DP / 8; ++jn) {
+        const int col = 8 * jn + 2 * t;
+        if (col < g.d) {
+          *reinterpret_cast<uint32_t*>(o0 + col) = pack2(dk[jn][0], dk[jn][1]);
+          *reinterpret_cast<uint32_t*>(o1 + col) = pack2(dk[jn][2], dk[jn][3]);
+          *reinterpret_cast<uint32_t*>(o0 + g.C + col) = pack2(dv[jn][0], dv[jn][1]);
+          *reinterpret_cast<uint32_t*>(o1 + g.C + col) = pack2(dv[jn][2], dv[jn][3]);
+        }
+      }
+    }
+  }
+
+  // ---- gradient of the bias table: fold this CTA's summed dS through the relative-position map
+  if (L.dtable != nullptr) {
+    const int pa0 = p0 >> 3, pc0 = p0 & 7;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int rel = (pa0 + (e >> 1) - j + 7) * 15 + (pc0 - (2 * t + (e & 1)) + 7);
+        atomicAdd(hist + hl * 225 + rel, dsum[j][e]);
+      }
+    __syncthreads();
+    for (int e = tid; e < nh_u * 225; e += nt) atomicAdd(L.dtable + (e % 225) * g.nh + u.h0 + e / 225, hist[e]);
+  }
+}
+
+template <int DP>
+size_t fwd_smem(int nheads) { return (size_t)nheads * 3 * 64 * DP * 2 + (size_t)nheads * 225 * 4 + 64 * 4 + 64 + 128; }
+template <int DP>
+size_t bwd_smem(int nheads) {
+  return (size_t)nheads * 4 * 64 * DP * 2 + (size_t)nheads * 2 * 8192 + (size_t)nheads * (2 * 225 + 64) * 4 + 64 * 4 + 64 + 128;
+}
+
+template <int DP>
+int launch_fwd_t(const AttnLaunch& L, cudaStream_t st) {
+  int maxh = 0;
+  for (int i = 0; i < L.nunits; ++i) maxh = L.u[i].nheads > maxh ? L.u[i].nheads : maxh;
+  const size_t smem = fwd_smem<DP>(maxh);
+  if (cudaFuncSetAttribute(attn_fwd_kernel<DP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return check_launch();
+  { KernelScope ks_("attn_fwd", st);
+    attn_fwd_kernel<DP><<<dim3((unsigned)L.geo.n_windows, L.nunits), maxh * 128, smem, st>>>(L); }
+  return check_launch();
+}
+
+template <int DP>
+int launch_bwd_t(const AttnLaunch& L, cudaStream_t st) {
+  int maxh = 0;
+  for (int i = 0; i < L.nunits; ++i) maxh = L.u[i].nheads > maxh ? L.u[i].nheads : maxh;
+  const size_t smem = bwd_smem<DP>(maxh);
+  if (cudaFuncSetAttribute(attn_bwd_kernel<DP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return check_launch();
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int per_sm = smem * 2 <= 220 * 1024 ? 2 : 1;
+  long long gx = (long long)sms * per_sm / L.nunits;
+  if (gx < 1) gx = 1;
+  if (gx > L.geo.n_windows) gx = L.geo.n_windows;
+  { KernelScope ks_("attn_bwd", st);
+    attn_bwd_kernel<DP><<<dim3((unsigned)gx, L.nunits), maxh * 128, smem, st>>>(L); }
+  return check_launch();
+}
+
+}  // namespace
+
+int launch_attn_fwd(const AttnLaunch& L, cudaStream_t st) {
+  return L.geo.dp == 32 ? launch_fwd_t<32>(L, st) : launch_fwd_t<16>(L, st);
+}
+int launch_attn_bwd(const AttnLaunch& L, cudaStream_t st) {
+  return L.geo.dp == 32 ? launch_bwd_t<32>(L, st) : launch_bwd_t<16>(L, st);
+}
+
+}  // namespace gswa

@@ -32,6 +32,7 @@ def run_gpu(cfg: LayerConfig, inp: dict, flags: int = 0, backward: bool = True, 
     b_qkv = dev["b_qkv"] if use_bias else None
     b_proj = dev["b_proj"] if use_bias else None
     gb.gswa_forward(desc, dev["x"], dev["w_qkv"], b_qkv, dev["w_proj"], b_proj, dev["bias_table"], y, saved, scratch)
+    gb.gswa_scratch_status(desc, scratch)
     out = {"y": y.float().cpu().numpy().astype(np.float64)}
     if backward and not inference:
         C, M, nh = cfg.C, cfg.window, cfg.num_heads
@@ -41,6 +42,7 @@ def run_gpu(cfg: LayerConfig, inp: dict, flags: int = 0, backward: bool = True, 
              "dbias_table": torch.full(((2 * M - 1) ** 2, nh), 7.0, device="cuda")}
         gb.gswa_backward(desc, dev["x"], dev["w_qkv"], b_qkv, dev["w_proj"], dev["bias_table"], saved, dev["dy"],
                          g["dx"], g["dw_qkv"], g["db_qkv"], g["dw_proj"], g["db_proj"], g["dbias_table"], scratch)
+        gb.gswa_scratch_status(desc, scratch)
         for k, v in g.items():
             out[k] = v.float().cpu().numpy().astype(np.float64)
     torch.cuda.synchronize()
