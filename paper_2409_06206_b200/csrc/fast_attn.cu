@@ -156,85 +156,103 @@ __device__ __forceinline__ void bias_and_mask(float (*s)[4], const float* tab, c
 }
 
 // ------------------------------------------------------------------------------------------
-// forward: one CTA per (window, unit); 4 warps per head, 16 query rows per warp
+// forward: persistent CTAs stride over the windows of a unit; 4 warps per head, 16 query rows per
+// warp.  The q,k,v tiles of the next window are copied into the second buffer while the current
+// window is being computed.
 // ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void cp_async_wait_1() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+
 template <int DP>
-__global__ void __launch_bounds__(512) attn_fwd_kernel(const __grid_constant__ AttnLaunch L) {
+__global__ void __launch_bounds__(384, 2) attn_fwd_kernel(const __grid_constant__ AttnLaunch L) {
   const AttnUnit& u = L.u[blockIdx.y];
   const FastGeom& g = L.geo;
   extern __shared__ __align__(128) unsigned char sm[];
   const int nh_u = u.nheads;
-  unsigned char* tiles = sm;
-  float* tab = reinterpret_cast<float*>(tiles + (size_t)nh_u * 3 * 64 * DP * 2);
-  int* tok = reinterpret_cast<int*>(tab + nh_u * 225);
-  unsigned char* reg = reinterpret_cast<unsigned char*>(tok + 64);
+  const int tile_bytes = nh_u * 3 * 64 * DP * 2;
+  float* tab = reinterpret_cast<float*>(sm + 2 * (size_t)tile_bytes);
+  int* tok2 = reinterpret_cast<int*>(tab + nh_u * 225);
+  unsigned char* reg2 = reinterpret_cast<unsigned char*>(tok2 + 128);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nt = nh_u * 128;
   if (tid >= nt) return;
-  const long long win = blockIdx.x;
 
-  load_tiles<DP>(tiles, L.qkv + u.qkv_off + win * u.qkv_wstride, nh_u * 3, tid, nt);
   for (int e = tid; e < nh_u * 225; e += nt)
     tab[e] = __bfloat162float(L.table[(e % 225) * g.nh + u.h0 + e / 225]);
-  const WinCtx wc = window_setup(g, u.s, win, tok, reg, tid);
-  cp_async_wait_all();
-  __syncthreads();
-
   const int hl = warp >> 2, r0 = (warp & 3) * 16, gq = lane >> 2, t = lane & 3;
-  const uint32_t q_base = smem_u32(tiles + (size_t)(hl * 3 + 0) * 64 * DP * 2);
-  const uint32_t k_base = q_base + 64 * DP * 2, v_base = k_base + 64 * DP * 2;
-  float s[8][4];
-  qk_scores<DP>(s, q_base, k_base, r0, lane);
   const int p0 = r0 + gq;
-  bias_and_mask(s, tab + hl * 225, reg, wc.masked, p0, t);
-
-  float m0 = -INFINITY, m1 = -INFINITY;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    m0 = fmaxf(m0, fmaxf(s[j][0], s[j][1]));
-    m1 = fmaxf(m1, fmaxf(s[j][2], s[j][3]));
-  }
-  m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1));
-  m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
-  m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1));
-  m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
-  float sum0 = 0.f, sum1 = 0.f;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    s[j][0] = exp2f(s[j][0] - m0);
-    s[j][1] = exp2f(s[j][1] - m0);
-    s[j][2] = exp2f(s[j][2] - m1);
-    s[j][3] = exp2f(s[j][3] - m1);
-    sum0 += s[j][0] + s[j][1];
-    sum1 += s[j][2] + s[j][3];
-  }
-  sum0 += __shfl_xor_sync(0xffffffffu, sum0, 1);
-  sum0 += __shfl_xor_sync(0xffffffffu, sum0, 2);
-  sum1 += __shfl_xor_sync(0xffffffffu, sum1, 1);
-  sum1 += __shfl_xor_sync(0xffffffffu, sum1, 2);
-
-  float o[DP / 8][4];
-#pragma unroll
-  for (int j = 0; j < DP / 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
-  regs_times_tile<DP>(o, s, v_base, lane);
-
-  const float inv0 = 1.f / sum0, inv1 = 1.f / sum1;
   const int h = u.h0 + hl;
-  __nv_bfloat16* out0 = L.A + (long long)tok[p0] * g.C + h * g.d;
-  __nv_bfloat16* out1 = L.A + (long long)tok[p0 + 8] * g.C + h * g.d;
+
+  long long win = blockIdx.x;
+  if (win < g.n_windows) load_tiles<DP>(sm, L.qkv + u.qkv_off + win * u.qkv_wstride, nh_u * 3, tid, nt);
+  cp_async_commit();
+  for (int buf = 0; win < g.n_windows; win += gridDim.x, buf ^= 1) {
+    const long long nxt = win + gridDim.x;
+    if (nxt < g.n_windows)
+      load_tiles<DP>(sm + (size_t)(buf ^ 1) * tile_bytes, L.qkv + u.qkv_off + nxt * u.qkv_wstride, nh_u * 3, tid, nt);
+    cp_async_commit();
+    int* tok = tok2 + buf * 64;
+    unsigned char* reg = reg2 + buf * 64;
+    const WinCtx wc = window_setup(g, u.s, win, tok, reg, tid);
+    cp_async_wait_1();
+    __syncthreads();
+
+    unsigned char* tiles = sm + (size_t)buf * tile_bytes;
+    const uint32_t q_base = smem_u32(tiles + (size_t)(hl * 3 + 0) * 64 * DP * 2);
+    const uint32_t k_base = q_base + 64 * DP * 2, v_base = k_base + 64 * DP * 2;
+    float s[8][4];
+    qk_scores<DP>(s, q_base, k_base, r0, lane);
+    bias_and_mask(s, tab + hl * 225, reg, wc.masked, p0, t);
+
+    float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-  for (int jn = 0; jn < DP / 8; ++jn) {
-    const int col = 8 * jn + 2 * t;
-    if (col < g.d) {
-      *reinterpret_cast<uint32_t*>(out0 + col) = pack2(o[jn][0] * inv0, o[jn][1] * inv0);
-      *reinterpret_cast<uint32_t*>(out1 + col) = pack2(o[jn][2] * inv1, o[jn][3] * inv1);
+    for (int j = 0; j < 8; ++j) {
+      m0 = fmaxf(m0, fmaxf(s[j][0], s[j][1]));
+      m1 = fmaxf(m1, fmaxf(s[j][2], s[j][3]));
     }
+    m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1));
+    m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
+    m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1));
+    m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
+    float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      s[j][0] = exp2f(s[j][0] - m0);
+      s[j][1] = exp2f(s[j][1] - m0);
+      s[j][2] = exp2f(s[j][2] - m1);
+      s[j][3] = exp2f(s[j][3] - m1);
+      sum0 += s[j][0] + s[j][1];
+      sum1 += s[j][2] + s[j][3];
+    }
+    sum0 += __shfl_xor_sync(0xffffffffu, sum0, 1);
+    sum0 += __shfl_xor_sync(0xffffffffu, sum0, 2);
+    sum1 += __shfl_xor_sync(0xffffffffu, sum1, 1);
+    sum1 += __shfl_xor_sync(0xffffffffu, sum1, 2);
+
+    float o[DP / 8][4];
+#pragma unroll
+    for (int j = 0; j < DP / 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
+    regs_times_tile<DP>(o, s, v_base, lane);
+
+    const float inv0 = 1.f / sum0, inv1 = 1.f / sum1;
+    __nv_bfloat16* out0 = L.A + (long long)tok[p0] * g.C + h * g.d;
+    __nv_bfloat16* out1 = L.A + (long long)tok[p0 + 8] * g.C + h * g.d;
+#pragma unroll
+    for (int jn = 0; jn < DP / 8; ++jn) {
+      const int col = 8 * jn + 2 * t;
+      if (col < g.d) {
+        *reinterpret_cast<uint32_t*>(out0 + col) = pack2(o[jn][0] * inv0, o[jn][1] * inv0);
+        *reinterpret_cast<uint32_t*>(out1 + col) = pack2(o[jn][2] * inv1, o[jn][3] * inv1);
+      }
+    }
+    if (L.Lt != nullptr && t == 0) {
+      float* lt = L.Lt + u.l_off + win * u.l_wstride + hl * 64;
+      lt[p0] = m0 * kLn2 + logf(sum0);
+      lt[p0 + 8] = m1 * kLn2 + logf(sum1);
+    }
+    __syncthreads();   // every warp is done with this buffer before the next iteration refills it
   }
-  if (L.Lt != nullptr && t == 0) {
-    float* lt = L.Lt + u.l_off + win * u.l_wstride + hl * 64;
-    lt[p0] = m0 * kLn2 + logf(sum0);
-    lt[p0 + 8] = m1 * kLn2 + logf(sum1);
-  }
+  cp_async_wait_all();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -247,15 +265,14 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
   extern __shared__ __align__(128) unsigned char sm[];
   const int nh_u = u.nheads;
   constexpr int kTile = 64 * DP * 2;
-  unsigned char* tiles = sm;                                   // q,k,v per head
-  unsigned char* dot = tiles + (size_t)nh_u * 3 * kTile;       // dO per head
-  unsigned char* Ps = dot + (size_t)nh_u * kTile;              // [head][64][64] bf16
+  const int in_bytes = nh_u * 4 * kTile;                       // q,k,v per head then dO per head: one window
+  unsigned char* Ps = sm + 2 * (size_t)in_bytes;               // [head][64][64] bf16
   unsigned char* dSs = Ps + (size_t)nh_u * 8192;
-  float* tab = reinterpret_cast<float*>(dSs + (size_t)nh_u * 8192);
+  float* Lrow2 = reinterpret_cast<float*>(dSs + (size_t)nh_u * 8192);   // [2][head][64], 16-byte aligned
+  float* tab = Lrow2 + 2 * nh_u * 64;
   float* hist = tab + nh_u * 225;
-  float* Lrow = hist + nh_u * 225;
-  int* tok = reinterpret_cast<int*>(Lrow + nh_u * 64);
-  unsigned char* reg = reinterpret_cast<unsigned char*>(tok + 64);
+  int* tok2 = reinterpret_cast<int*>(hist + nh_u * 225);       // [2][64]
+  unsigned char* reg2 = reinterpret_cast<unsigned char*>(tok2 + 128);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nt = nh_u * 128;
   if (tid >= nt) return;
@@ -266,9 +283,6 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
   }
   const int hl = warp >> 2, r0 = (warp & 3) * 16, gq = lane >> 2, t = lane & 3;
   const int h = u.h0 + hl;
-  const uint32_t q_base = smem_u32(tiles + (size_t)(hl * 3) * kTile);
-  const uint32_t k_base = q_base + kTile, v_base = k_base + kTile;
-  const uint32_t do_base = smem_u32(dot + (size_t)hl * kTile);
   unsigned char* Ph = Ps + (size_t)hl * 8192;
   unsigned char* dSh = dSs + (size_t)hl * 8192;
   const int p0 = r0 + gq;
@@ -276,14 +290,33 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
 #pragma unroll
   for (int j = 0; j < 8; ++j) dsum[j][0] = dsum[j][1] = dsum[j][2] = dsum[j][3] = 0.f;
 
-  for (long long win = blockIdx.x; win < g.n_windows; win += gridDim.x) {
-    __syncthreads();   // previous window's tiles, P and dS are no longer read
-    load_tiles<DP>(tiles, L.qkv + u.qkv_off + win * u.qkv_wstride, nh_u * 3, tid, nt);
-    load_tiles<DP>(dot, L.dO + u.do_off + win * u.do_wstride, nh_u, tid, nt);
-    for (int e = tid; e < nh_u * 64; e += nt) Lrow[e] = L.Lt[u.l_off + win * u.l_wstride + e];
+  // copies of one window's inputs into buffer `b` (asynchronous)
+  auto fetch = [&](long long w, int b) {
+    unsigned char* dst = sm + (size_t)b * in_bytes;
+    load_tiles<DP>(dst, L.qkv + u.qkv_off + w * u.qkv_wstride, nh_u * 3, tid, nt);
+    load_tiles<DP>(dst + (size_t)nh_u * 3 * kTile, L.dO + u.do_off + w * u.do_wstride, nh_u, tid, nt);
+    const float* lsrc = L.Lt + u.l_off + w * u.l_wstride;
+    float* ldst = Lrow2 + b * nh_u * 64;
+    for (int e = tid; e < nh_u * 16; e += nt) cp_async16(smem_u32(ldst + 4 * e), lsrc + 4 * e);
+  };
+
+  long long win = blockIdx.x;
+  if (win < g.n_windows) fetch(win, 0);
+  cp_async_commit();
+  for (int buf = 0; win < g.n_windows; win += gridDim.x, buf ^= 1) {
+    const long long nxt = win + gridDim.x;
+    if (nxt < g.n_windows) fetch(nxt, buf ^ 1);
+    cp_async_commit();
+    int* tok = tok2 + buf * 64;
+    unsigned char* reg = reg2 + buf * 64;
+    const float* Lrow = Lrow2 + buf * nh_u * 64;
     const WinCtx wc = window_setup(g, u.s, win, tok, reg, tid);
-    cp_async_wait_all();
+    cp_async_wait_1();
     __syncthreads();
+    unsigned char* tiles = sm + (size_t)buf * in_bytes;
+    const uint32_t q_base = smem_u32(tiles + (size_t)(hl * 3) * kTile);
+    const uint32_t k_base = q_base + kTile, v_base = k_base + kTile;
+    const uint32_t do_base = smem_u32(tiles + (size_t)(nh_u * 3 + hl) * kTile);
 
     // ---- query-major phase: this warp owns query rows r0 .. r0+15 of head hl
     float s[8][4];
@@ -382,7 +415,9 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
         }
       }
     }
+    __syncthreads();   // tiles, P and dS of this window are no longer read
   }
+  cp_async_wait_all();
 
   // ---- gradient of the bias table: fold this CTA's summed dS through the relative-position map
   if (L.dtable != nullptr) {
@@ -400,10 +435,10 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
 }
 
 template <int DP>
-size_t fwd_smem(int nheads) { return (size_t)nheads * 3 * 64 * DP * 2 + (size_t)nheads * 225 * 4 + 64 * 4 + 64 + 128; }
+size_t fwd_smem(int nheads) { return (size_t)2 * nheads * 3 * 64 * DP * 2 + (size_t)nheads * 225 * 4 + 128 * 4 + 128 + 128; }
 template <int DP>
 size_t bwd_smem(int nheads) {
-  return (size_t)nheads * 4 * 64 * DP * 2 + (size_t)nheads * 2 * 8192 + (size_t)nheads * (2 * 225 + 64) * 4 + 64 * 4 + 64 + 128;
+  return (size_t)2 * nheads * 4 * 64 * DP * 2 + (size_t)nheads * 2 * 8192 + (size_t)nheads * (2 * 225 + 2 * 64) * 4 + 128 * 4 + 128 + 128;
 }
 
 template <int DP>
@@ -413,8 +448,15 @@ int launch_fwd_t(const AttnLaunch& L, cudaStream_t st) {
   const size_t smem = fwd_smem<DP>(maxh);
   if (cudaFuncSetAttribute(attn_fwd_kernel<DP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return check_launch();
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int per_sm = smem * 2 <= 220 * 1024 ? 2 : 1;
+  long long gx = (long long)sms * per_sm / L.nunits;
+  if (gx < 1) gx = 1;
+  if (gx > L.geo.n_windows) gx = L.geo.n_windows;
   { KernelScope ks_("attn_fwd", st);
-    attn_fwd_kernel<DP><<<dim3((unsigned)L.geo.n_windows, L.nunits), maxh * 128, smem, st>>>(L); }
+    attn_fwd_kernel<DP><<<dim3((unsigned)gx, L.nunits), maxh * 128, smem, st>>>(L); }
   return check_launch();
 }
 

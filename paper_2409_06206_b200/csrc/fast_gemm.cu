@@ -40,16 +40,26 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatil
   if (err) atomicExch(err, 1);
   return false;
 }
-// All lanes of a warp take the same decision.
+// Warp-wide wait: one lane polls (32 lanes polling one barrier word only serialise on it), the
+// outcome is broadcast, and the warp barrier orders the other lanes after the observation.
 __device__ __forceinline__ bool wait_bar_warp(uint64_t* bar, uint32_t parity, volatile int* abort_s, int* err) {
-  const bool ok = wait_bar(bar, parity, abort_s, err);
-  return __all_sync(0xffffffffu, ok);
+  int ok = 1;
+  if ((threadIdx.x & 31) == 0) ok = wait_bar(bar, parity, abort_s, err) ? 1 : 0;
+  ok = __shfl_sync(0xffffffffu, ok, 0);
+  return ok != 0;
+}
+
+// A loader warp publishes a stage: every lane has waited for its own copies; the proxy fence makes
+// them visible to the tensor core, the warp barrier orders the lanes, one lane arrives.
+__device__ __forceinline__ void publish(uint64_t* bar, int lane) {
+  fence_proxy_async();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bar);
 }
 
 __device__ __forceinline__ unsigned char* align1024(unsigned char* p) {
   return reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~(uintptr_t)1023);
 }
-__device__ __forceinline__ uint2 ldg8(const __nv_bfloat16* p) { return __ldg(reinterpret_cast<const uint2*>(p)); }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -85,8 +95,8 @@ __global__ void __launch_bounds__(kThreads, 1) gw_kernel(const __grid_constant__
   fence_proxy_async();
   if (tid == 0) {
     abort_s = 0;
-    for (int i = 0; i < 2; ++i) { mbar_init(&full[i], kLoadThreads); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 8; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], 128); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&full[i], kLoadWarps); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < 8; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], kEpiWarps); }
     mbar_init_fence();
   }
   const uint32_t tcols = pow2_cols(NT);
@@ -98,50 +108,62 @@ __global__ void __launch_bounds__(kThreads, 1) gw_kernel(const __grid_constant__
   const long long n_tiles = (u.n_windows + 1) / 2;
 
   if (warp > kEpiWarps) {
-    // ---------------- loaders: warp lw owns window column lw of every window row
+    // ---------------- loaders: warp lw owns window column lw of every window row.  Asynchronous
+    // 8-byte copies land directly in the swizzled operand image; a stage is published one tile
+    // late (after its copies have completed), so two tiles of loads are in flight per SM.
     const int lw = warp - kEpiWarps - 1;
     constexpr int NPC = (CP / 4 + 31) / 32;      // 8-byte pieces per lane per row
+    // Per-lane constants: tile row r = lw + 8*(8*half + a) has (r & 7) == lw, so the swizzled
+    // destination of a piece is a fixed offset plus 1024 bytes per row step.
+    uint32_t dst0[NPC];
+    int colb[NPC];                                // byte offset of the piece inside a source row, -1 = padding
+#pragma unroll
+    for (int pi = 0; pi < NPC; ++pi) {
+      const int col = (lane + 32 * pi) * 4;
+      dst0[pi] = (uint32_t)((col >> 6) * kAtomBytesA) + sw128_offset(lw, col & 63);
+      colb[pi] = col < u.kvalid ? col * 2 : -1;
+    }
+    const char* const srcA = reinterpret_cast<const char*>(u.A);
+    const long long row_bytes = (long long)u.lda * 2;
     int it = 0;
     for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
       const int stage = it & 1;
       if (!wait_bar_warp(&empty[stage], ((it >> 1) & 1) ^ 1, &abort_s, L.err)) break;
-      unsigned char* sA = sA0 + stage * kStageBytes;
+      const uint32_t sA = smem_u32(sA0 + stage * kStageBytes);
 #pragma unroll
-      for (int kb = 0; kb < 16; kb += 4) {
-        uint2 v[4][NPC];
+      for (int half = 0; half < 2; ++half) {
+        // one window of the pair: cyclic shift + partition are this address arithmetic
+        const int win = 2 * (int)tile + half;
+        const bool wv = win < (int)u.n_windows;
+        const int b = win / u.nW, w = win - b * u.nW;
+        const int wi = w / u.nWw, wj = w - wi * u.nWw;
+        int j = wj * 8 + lw + u.s;
+        if (j >= u.W) j -= u.W;
+        const int i0 = wi * 8 + u.s;
+        const char* col0 = srcA + ((long long)b * u.H * u.W + j) * row_bytes;
+        const long long line_bytes = (long long)u.W * row_bytes;
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          const int k = kb + kk;
-          const long long win = 2 * tile + (k >> 3);
-          const __nv_bfloat16* src = nullptr;
-          if (win < u.n_windows) {
-            const int b = (int)(win / u.nW), w = (int)(win % u.nW);
-            int i = (w / u.nWw) * 8 + (k & 7) + u.s, j = (w % u.nWw) * 8 + lw + u.s;
-            if (i >= u.H) i -= u.H;
-            if (j >= u.W) j -= u.W;
-            src = u.A + ((long long)(b * u.H + i) * u.W + j) * u.lda;
-          }
-#pragma unroll
-          for (int pi = 0; pi < NPC; ++pi) {
-            const int col = (lane + 32 * pi) * 4;
-            v[kk][pi] = make_uint2(0u, 0u);
-            if (src != nullptr && col < u.kvalid) v[kk][pi] = ldg8(src + col);
-          }
-        }
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          const int r = lw + 8 * (kb + kk);
+        for (int a = 0; a < 8; ++a) {
+          int i = i0 + a;
+          if (i >= u.H) i -= u.H;
+          const char* src = col0 + i * line_bytes;
 #pragma unroll
           for (int pi = 0; pi < NPC; ++pi) {
-            const int col = (lane + 32 * pi) * 4;
-            if (col < CP)
-              *reinterpret_cast<uint2*>(sA + (col >> 6) * kAtomBytesA + sw128_offset(r, col & 63)) = v[kk][pi];
+            if ((lane + 32 * pi) * 4 < CP) {
+              const bool v = wv && colb[pi] >= 0;
+              cp_async8(sA + dst0[pi] + (8 * half + a) * 1024, v ? src + colb[pi] : srcA, v);
+            }
           }
         }
       }
-      fence_proxy_async();
-      mbar_arrive(&full[stage]);
+      cp_async_commit();
+      if (it > 0) {
+        cp_async_wait(1);
+        publish(&full[(it - 1) & 1], lane);
+      }
     }
+    cp_async_wait(0);
+    if (it > 0 && __all_sync(0xffffffffu, abort_s == 0)) publish(&full[(it - 1) & 1], lane);
   } else if (warp == kEpiWarps) {
     // ---------------- MMA issue
     if (lane == 0) {
@@ -200,7 +222,8 @@ __global__ void __launch_bounds__(kThreads, 1) gw_kernel(const __grid_constant__
           }
         }
         fence_before_sync();
-        mbar_arrive(&tempty[c]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty[c]);
       }
     }
   }
@@ -237,8 +260,8 @@ __global__ void __launch_bounds__(kThreads, 1) gt_kernel(const __grid_constant__
   fence_proxy_async();
   if (tid == 0) {
     abort_s = 0;
-    for (int i = 0; i < 8; ++i) { mbar_init(&full[i], kLoadThreads); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], 128); }
+    for (int i = 0; i < 8; ++i) { mbar_init(&full[i], kLoadWarps); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], kEpiWarps); }
     mbar_init_fence();
   }
   const uint32_t tcols = pow2_cols(2 * NB);
@@ -250,29 +273,53 @@ __global__ void __launch_bounds__(kThreads, 1) gt_kernel(const __grid_constant__
   const long long n_tiles = (L.rows + 127) / 128;
 
   if (warp > kEpiWarps) {
-    // ---------------- loaders: thread -> (8-byte piece of the atom, 8 rows)
+    // ---------------- loaders: thread -> (8-byte piece of the atom, 8 rows), asynchronous copies;
+    // a ring stage is published `lag` steps after it was issued, once its copies have landed.
     const int tl = tid - 32 * (kEpiWarps + 1);
     const int piece = tl & 15, row0 = tl >> 4;
-    int st = 0, ph = 0;
+    const int lag = S - 1 < 3 ? S - 1 : 3;
+    const uint32_t ringA = smem_u32(ring);
+    // rows row0 + 16k share (row & 7), so a piece's swizzled destination is dst0 + 2048 k
+    const uint32_t dst0 = sw128_offset(row0, piece * 4);
+    const char* const srcA = reinterpret_cast<const char*>(L.A);
+    const long long row_bytes = (long long)L.lda * 2;
+    int st = 0, ph = 0, n = 0, pub = 0;          // pub: ring stage of the oldest unpublished step
     bool ok = true;
     for (long long tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      const long long trow = tile * 128 + row0;
+      const char* const src_t = srcA + trow * row_bytes + piece * 8;
+      const bool full_tile = (tile + 1) * 128 <= L.rows;
       for (int atom = 0; atom < natoms; ++atom) {
         if (!wait_bar_warp(&empty[st], ph ^ 1, &abort_s, L.err)) { ok = false; break; }
-        const int col = atom * 64 + piece * 4;
-        uint2 v[8];
+        const bool cv = atom * 64 + piece * 4 < L.kvalid;
+        const uint32_t sA = ringA + st * kAtomStage + dst0;
+        const char* src = src_t + atom * 128;
+        if (full_tile) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const long long t = tile * 128 + row0 + 16 * k;
-          v[k] = make_uint2(0u, 0u);
-          if (t < L.rows && col < L.kvalid) v[k] = ldg8(L.A + t * L.lda + col);
+          for (int k = 0; k < 8; ++k) cp_async8(sA + k * 2048, cv ? src + k * 16 * row_bytes : srcA, cv);
+        } else {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const bool v = cv && trow + 16 * k < L.rows;
+            cp_async8(sA + k * 2048, v ? src + k * 16 * row_bytes : srcA, v);
+          }
         }
-        unsigned char* sA = ring + st * kAtomStage;
-#pragma unroll
-        for (int k = 0; k < 8; ++k)
-          *reinterpret_cast<uint2*>(sA + sw128_offset(row0 + 16 * k, piece * 4)) = v[k];
-        fence_proxy_async();
-        mbar_arrive(&full[st]);
+        cp_async_commit();
         if (++st == S) { st = 0; ph ^= 1; }
+        if (++n > lag) {
+          cp_async_wait(lag);
+          publish(&full[pub], lane);
+          if (++pub == S) pub = 0;
+        }
+      }
+    }
+    {
+      int left = n < lag ? n : lag;              // steps issued but not yet published
+      while (left > 0) {
+        cp_async_wait(left - 1);
+        if (ok) publish(&full[pub], lane);
+        if (++pub == S) pub = 0;
+        --left;
       }
     }
   } else if (warp == kEpiWarps) {
@@ -313,23 +360,33 @@ __global__ void __launch_bounds__(kThreads, 1) gt_kernel(const __grid_constant__
         uint32_t v[32];
         tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + buf * NB + c0, v);
         tmem_ld_wait();
-        uint32_t* dst = reinterpret_cast<uint32_t*>(mystg + ((size_t)lane * ncols + c0) * 2);
+        // the lane's row of the staging tile; rows are 2*ncols bytes apart (a multiple of 8, and an
+        // odd multiple for C = 180, so these 8-byte stores do not collide on banks)
+        uint2* dst = reinterpret_cast<uint2*>(mystg + ((size_t)lane * ncols + c0) * 2);
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-          if (c0 + 2 * j < ncols)
-            dst[j] = pack_bf16(__uint_as_float(v[2 * j]) + sBias[c0 + 2 * j],
-                               __uint_as_float(v[2 * j + 1]) + sBias[c0 + 2 * j + 1]);
+        for (int j = 0; j < 8; ++j)
+          if (c0 + 4 * j < ncols)
+            dst[j] = make_uint2(pack_bf16(__uint_as_float(v[4 * j]) + sBias[c0 + 4 * j],
+                                          __uint_as_float(v[4 * j + 1]) + sBias[c0 + 4 * j + 1]),
+                                pack_bf16(__uint_as_float(v[4 * j + 2]) + sBias[c0 + 4 * j + 2],
+                                          __uint_as_float(v[4 * j + 3]) + sBias[c0 + 4 * j + 3]));
       }
       fence_before_sync();
-      mbar_arrive(&tempty[buf]);
       __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty[buf]);
+      // copy-out: lane = 8-byte piece of a row (two pieces per lane cover up to 256 columns)
       const long long trow0 = tile * 128 + warp * 32;
-      for (int e = lane; e < 32 * n8; e += 32) {
-        const int rr = e / n8, pc = e - rr * n8;
-        const long long t = trow0 + rr;
-        if (t < L.rows)
-          *reinterpret_cast<uint2*>(L.out + t * L.ldo + sp.col0 + pc * 4) =
-              *reinterpret_cast<const uint2*>(mystg + ((size_t)rr * ncols + pc * 4) * 2);
+      const int nrows = L.rows - trow0 < 32 ? (int)(L.rows - trow0) : 32;
+      char* const obase = reinterpret_cast<char*>(L.out + trow0 * L.ldo + sp.col0) + lane * 8;
+      const long long obytes = (long long)L.ldo * 2;
+      const unsigned char* sbase = mystg + lane * 8;
+      const bool p0 = lane < n8, p1 = lane + 32 < n8;
+#pragma unroll 4
+      for (int rr = 0; rr < nrows; ++rr) {
+        if (p0) *reinterpret_cast<uint2*>(obase + rr * obytes) = *reinterpret_cast<const uint2*>(sbase + rr * ncols * 2);
+        if (p1)
+          *reinterpret_cast<uint2*>(obase + rr * obytes + 256) =
+              *reinterpret_cast<const uint2*>(sbase + rr * ncols * 2 + 256);
       }
       __syncwarp();
     }
@@ -371,7 +428,7 @@ __global__ void __launch_bounds__(kThreads, 1) gr_kernel(const __grid_constant__
 
   if (tid == 0) {
     abort_s = 0;
-    for (int i = 0; i < S; ++i) { mbar_init(&full[i], kLoadThreads); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < S; ++i) { mbar_init(&full[i], kLoadWarps); mbar_init(&empty[i], 1); }
     mbar_init(&done, 1);
     mbar_init_fence();
   }
@@ -385,45 +442,74 @@ __global__ void __launch_bounds__(kThreads, 1) gr_kernel(const __grid_constant__
   if (warp > kEpiWarps) {
     const int lw = warp - kEpiWarps - 1;
     const int lcol = mb * 128 + lane * 4;
-    int st = 0, ph = 0;
+    constexpr int lag = 2;
+    // Stage row r = lw + 8k has (r & 7) == lw: every piece's swizzled destination is a per-lane
+    // constant plus 1024 bytes per k.  Pieces that never change (K/M padding, the ones column that
+    // turns the GEMM into a column sum of L) are written once per stage buffer, before the loop.
+    const uint32_t dL = (uint32_t)((lane >> 4) * 8192) + sw128_offset(lw, (lane & 15) * 4);
+    const bool lvalid = lcol < L.mvalid;
+    uint32_t dR[2];
+    int rkind[2];                                 // 0 = data, 1 = ones column, 2 = zero padding, 3 = outside the stage
+#pragma unroll
+    for (int pi = 0; pi < 2; ++pi) {
+      const int col = (lane + 32 * pi) * 4;
+      dR[pi] = (uint32_t)(2 * 8192 + (col >> 6) * 8192) + sw128_offset(lw, col & 63);
+      rkind[pi] = col >= NP ? 3 : (col < L.nvalid ? 0 : (col == L.nvalid ? 1 : 2));
+    }
+    for (int sgi = 0; sgi < S; ++sgi) {
+      unsigned char* base = sm + (size_t)sgi * stage_bytes;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        if (!lvalid) *reinterpret_cast<uint2*>(base + dL + k * 1024) = make_uint2(0u, 0u);
+#pragma unroll
+        for (int pi = 0; pi < 2; ++pi)
+          if (rkind[pi] == 1 || rkind[pi] == 2)
+            *reinterpret_cast<uint2*>(base + dR[pi] + k * 1024) = make_uint2(rkind[pi] == 1 ? 0x3F80u : 0u, 0u);
+      }
+    }
+    const char* const srcL = reinterpret_cast<const char*>(L.L);
+    const char* const srcR = reinterpret_cast<const char*>(L.R);
+    const long long lrow = (long long)L.ldl * 2, rrow = (long long)L.ldr * 2;
+    int st = 0, ph = 0, n = 0, pub = 0;
+    bool ok = true;
     for (int s = 0; s < nst; ++s) {
-      if (!wait_bar_warp(&empty[st], ph ^ 1, &abort_s, L.err)) break;
-      unsigned char* sL = sm + (size_t)st * stage_bytes;
-      unsigned char* sR = sL + 2 * 8192;
-      const long long tb = t0 + (long long)s * 64;
+      if (!wait_bar_warp(&empty[st], ph ^ 1, &abort_s, L.err)) { ok = false; break; }
+      const uint32_t sS = smem_u32(sm + (size_t)st * stage_bytes);
+      const long long tb = t0 + (long long)s * 64 + lw;
+      const char* pl = srcL + tb * lrow + lcol * 2;
+      const char* pr = srcR + tb * rrow + lane * 8;
+      if (tb - lw + 64 <= t1) {
 #pragma unroll
-      for (int kb = 0; kb < 8; kb += 4) {
-        uint2 vl[4], vr[4][2];
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          const long long t = tb + lw + 8 * (kb + kk);
-          const bool tv = t < t1;
-          vl[kk] = make_uint2(0u, 0u);
-          if (tv && lcol < L.mvalid) vl[kk] = ldg8(L.L + t * L.ldl + lcol);
-#pragma unroll
-          for (int pi = 0; pi < 2; ++pi) {
-            const int col = (lane + 32 * pi) * 4;
-            vr[kk][pi] = make_uint2(0u, 0u);
-            if (tv) {
-              if (col < L.nvalid) vr[kk][pi] = ldg8(L.R + t * L.ldr + col);
-              else if (col == L.nvalid) vr[kk][pi] = make_uint2(0x3F80u, 0u);   // bf16 1.0: the ones column
-            }
-          }
+        for (int k = 0; k < 8; ++k) {
+          if (lvalid) cp_async8(sS + dL + k * 1024, pl + k * 8 * lrow, true);
+          if (rkind[0] == 0) cp_async8(sS + dR[0] + k * 1024, pr + k * 8 * rrow, true);
+          if (rkind[1] == 0) cp_async8(sS + dR[1] + k * 1024, pr + k * 8 * rrow + 256, true);
         }
+      } else {
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          const int r = lw + 8 * (kb + kk);
-          *reinterpret_cast<uint2*>(sL + (lane >> 4) * 8192 + sw128_offset(r, (lane & 15) * 4)) = vl[kk];
-#pragma unroll
-          for (int pi = 0; pi < 2; ++pi) {
-            const int col = (lane + 32 * pi) * 4;
-            if (col < NP) *reinterpret_cast<uint2*>(sR + (col >> 6) * 8192 + sw128_offset(r, col & 63)) = vr[kk][pi];
-          }
+        for (int k = 0; k < 8; ++k) {
+          const bool tv = tb + 8 * k < t1;
+          if (lvalid) cp_async8(sS + dL + k * 1024, tv ? pl + k * 8 * lrow : srcL, tv);
+          if (rkind[0] == 0) cp_async8(sS + dR[0] + k * 1024, tv ? pr + k * 8 * rrow : srcR, tv);
+          if (rkind[1] == 0) cp_async8(sS + dR[1] + k * 1024, tv ? pr + k * 8 * rrow + 256 : srcR, tv);
         }
       }
-      fence_proxy_async();
-      mbar_arrive(&full[st]);
+      cp_async_commit();
       if (++st == S) { st = 0; ph ^= 1; }
+      if (++n > lag) {
+        cp_async_wait(lag);
+        publish(&full[pub], lane);
+        if (++pub == S) pub = 0;
+      }
+    }
+    {
+      int left = n < lag ? n : lag;
+      while (left > 0) {
+        cp_async_wait(left - 1);
+        if (ok) publish(&full[pub], lane);
+        if (++pub == S) pub = 0;
+        --left;
+      }
     }
   } else if (warp == kEpiWarps) {
     if (lane == 0) {
