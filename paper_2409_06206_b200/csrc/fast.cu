@@ -28,8 +28,9 @@ int heads_per_unit(int Cp, int dp) {
   int best = 0;
   for (int n = 1; n <= 3; ++n) {
     const size_t NT = (size_t)n * 3 * dp;
-    const size_t smem = 1024 + NT * Cp * 2 + (size_t)2 * 128 * Cp * 2 + NT * 4 + 64;
-    if (smem <= kSmemBudget + 8 * 1024 && NT <= 512) best = n;
+    const int slots = Cp / 64 + 1 > 4 ? Cp / 64 + 1 : 4;
+    const size_t smem = 1024 + NT * Cp * 2 + 8 * 2 * 32 * dp * 2 + (size_t)slots * 128 * 128 + NT * 4 + 64;   // weights, staging, ring
+    if (smem <= kSmemBudget && NT <= 512) best = n;
   }
   return best;
 }
@@ -54,7 +55,7 @@ bool token_split(int C, int kvalid, TokenSplit* ts) {
     const int NB = (int)align_up((size_t)(C + nsplit - 1) / nsplit, 32);
     if (NB > 256) continue;
     const size_t fixed = 1024 + (size_t)natoms * NB * 128 + (size_t)128 * NB * 2 + NB * 4 + 64;
-    if (fixed + 3 * 16384 > kSmemBudget) continue;
+    if (fixed + 4 * 16384 > kSmemBudget) continue;
     int S = (int)((kSmemBudget - fixed) / 16384);
     if (S > 8) S = 8;
     *ts = TokenSplit{(C + NB - 1) / NB, NB, S, natoms};

@@ -8,6 +8,10 @@
 //   qkv tiles of group g : base + qkv_off[g] + window*(gh*3*64*DP) + ((hl*3 + kind)*64 + slot)*DP + c
 //   dO  tiles of group g : base + do_off[g]  + window*(gh*64*DP)   + (hl*64 + slot)*DP + c
 //   L   tiles of group g : base + l_off[g]   + window*(gh*64)      +  hl*64 + slot            (float)
+// Inside a [64][DP] block the 16-byte chunks of a row are permuted (tile_off below) so that the block
+// is at the same time the shared-memory image the attention kernels read with ldmatrix: the GEMM
+// epilogue builds the image in shared memory and ships it with one bulk copy, the attention kernels
+// fetch it with plain linear copies.
 // "Token-major" buffers are packed [T, cols] rows in original token order (attention output A[T,C],
 // dqkv[T,3C]); the attention epilogues undo partition and shift when they store into them.
 #pragma once
@@ -17,6 +21,15 @@
 namespace gswa {
 
 constexpr int kMaxUnits = 8;   // (group, head range) work units per launch
+
+// Byte offset of 16-byte chunk `chunk` of row `row` inside a [64][DP] bf16 tile image: eight
+// consecutive rows map to eight different 16-byte bank groups (ldmatrix and 16-byte stores of
+// consecutive rows are conflict free).
+template <int DP>
+__host__ __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
+  constexpr int CH = DP / 8;                // chunks per row (4 or 2)
+  return (uint32_t)(row * (DP * 2) + ((chunk ^ ((row / (8 / CH)) % CH)) << 4));
+}
 
 struct FastGeom {
   int B, H, W, C, nh, d, dp, G;
@@ -43,6 +56,7 @@ struct GWUnit {
 struct GWLaunch {
   GWUnit u[kMaxUnits];
   int* err;
+  int nslots;                  // ring slots of 16 KB (set by launch_gw)
 };
 
 // ---- token GEMM: rows in token order from packed [T, lda], output packed rows [T, ldo]

@@ -45,26 +45,16 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
 
 constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
 
-// Shared-memory image of a [64][DP] tile: 16-byte chunks of a row permuted so that ldmatrix of
-// eight consecutive rows is bank-conflict free.
-template <int DP>
-__device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
-  constexpr int CH = DP / 8;                // chunks per row (4 or 2)
-  return (uint32_t)(row * (DP * 2) + ((chunk ^ ((row / (8 / CH)) % CH)) << 4));
-}
 // [64][64] bf16 matrices (P, dS): 128-byte rows, chunk ^= row & 7.
 __device__ __forceinline__ uint32_t sq_off(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
 
+// Tiles arrive from global memory already in their shared-memory image (tile_off): a linear copy.
 template <int DP>
 __device__ __forceinline__ void load_tiles(unsigned char* dst, const __nv_bfloat16* src, int nblocks, int tid, int nt) {
-  constexpr int CH = DP / 8;
-  const int nchunks = nblocks * 64 * CH;
+  const int nchunks = nblocks * 64 * (DP / 8);
   const uint32_t d0 = smem_u32(dst);
-  for (int ci = tid; ci < nchunks; ci += nt) {
-    const int rowg = ci / CH, chunk = ci % CH;
-    cp_async16(d0 + (rowg >> 6) * (64 * DP * 2) + tile_off<DP>(rowg & 63, chunk),
-               reinterpret_cast<const unsigned char*>(src) + (size_t)ci * 16);
-  }
+  for (int ci = tid; ci < nchunks; ci += nt)
+    cp_async16(d0 + ci * 16, reinterpret_cast<const unsigned char*>(src) + (size_t)ci * 16);
 }
 
 // S (16 rows x 64 keys) = Q K^T for the warp's rows; returns accumulators in s[8][4].

@@ -23,8 +23,23 @@ using namespace umma;
 namespace {
 
 constexpr int kEpiWarps = 4, kLoadWarps = 8;
-constexpr int kThreads = 32 * (kEpiWarps + 1 + kLoadWarps);   // 416
-constexpr int kLoadThreads = 32 * kLoadWarps;                 // 256
+constexpr int kThreads = 32 * (kEpiWarps + 1 + kLoadWarps);   // 416 (gr_kernel)
+// gw_kernel / gt_kernel drain TMEM with two warps per 32-lane quadrant (a warp may only read the
+// TMEM lanes 32*(warp%4) .. +31): warps 0-7 epilogue, warp 8 MMA issue, warps 9-16 loaders.
+constexpr int kEpi2 = 8;
+constexpr int kThreads2 = 32 * (kEpi2 + 1 + kLoadWarps);      // 544
+__device__ __forceinline__ void pair_sync(int quad) { asm volatile("bar.sync %0, 64;" ::"r"(quad + 1) : "memory"); }
+// Barrier of the two warps of a quadrant that also ANDs a predicate, so that both take the same
+// decision to go on or to give up (a warp must never be left waiting for a partner that returned).
+__device__ __forceinline__ bool pair_vote(int quad, bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %2, 0;\n\tbar.red.and.pred p, %1, 64, q;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(r)
+      : "r"(quad + 1), "r"((uint32_t)ok)
+      : "memory");
+  return r != 0;
+}
 constexpr uint32_t kSpinLimit = 2000000u;
 
 // Bounded wait shared by all roles.  On timeout raises the CTA-wide abort flag and the error word.
@@ -71,165 +86,253 @@ __host__ __device__ inline uint32_t pow2_cols(int n) {
 }
 
 // ==========================================================================================
+// Shared producer / consumer pieces of gw_kernel and gt_kernel
+// ==========================================================================================
+// The A operand of both kernels is a 128-row tile cut into K atoms of 64 columns (16 KB each,
+// 128-byte swizzled rows) that travel through a ring of `S` shared-memory slots.  The eight loader
+// warps form four sets of two warps; set q fills ring steps q, q+4, q+8, ...: it waits until the
+// tensor core has released the slot, issues its asynchronous copies, waits for them to land, and
+// publishes the slot at once.  Four steps of loads are therefore in flight per SM and a slot becomes
+// visible to the MMA warp as soon as its own data has arrived.
+constexpr int kSets = 4;                      // loader sets
+constexpr int kAtomBytes = 128 * 128;         // one ring slot
+
+struct RingPos {
+  int slot, ph;                               // slot index and phase parity of ring step g
+  __device__ __forceinline__ void init(int g, int S) { slot = g % S; ph = (g / S) & 1; }
+  __device__ __forceinline__ void advance(int n, int S) {
+    slot += n;
+    while (slot >= S) { slot -= S; ph ^= 1; }
+  }
+};
+
+// One thread of a loader set: 8-token column `lw` of every 8-row group, 16-byte chunk `pp` of the atom
+// row (copied as two 8-byte pieces: source rows are only 8-byte aligned).  Tile row r = lw + 8k has
+// (r & 7) == lw, so the swizzled destination is dst0 + 1024 k.
+struct LoaderLane {
+  int lw, pp;
+  uint32_t dst0;
+  __device__ __forceinline__ void init(int ts) {
+    lw = ts & 7;
+    pp = ts >> 3;
+    dst0 = sw128_offset(lw, pp * 8);
+  }
+};
+
+// Barriers over the eight epilogue warps (hardware barrier 5, 256 threads); the voting form ANDs a
+// predicate so that all of them go on or give up together.
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 5, 256;" ::: "memory"); }
+__device__ __forceinline__ bool epi_vote(bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, 5, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(r)
+      : "r"((uint32_t)ok)
+      : "memory");
+  return r != 0;
+}
+// Bulk asynchronous copy shared -> global (sizes and addresses multiples of 16 bytes).
+__device__ __forceinline__ void bulk_store(void* gdst, uint32_t ssrc, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(ssrc), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// ==========================================================================================
 // gw_kernel
 // ==========================================================================================
 template <int CP, int DP>
-__global__ void __launch_bounds__(kThreads, 1) gw_kernel(const __grid_constant__ GWLaunch L) {
+__global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant__ GWLaunch L) {
   const GWUnit& u = L.u[blockIdx.y];
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = align1024(smem_raw);
-  constexpr int kStageBytes = 128 * CP * 2;
-  constexpr int kAtomBytesA = 128 * 128;
+  constexpr int NA = CP / 64;                  // K atoms per tile
   const int NT = u.nchunks * u.cw;
+  const int S = L.nslots;
   unsigned char* sB = sm;
-  unsigned char* sA0 = sB + (size_t)NT * CP * 2;
-  float* sBias = reinterpret_cast<float*>(sA0 + 2 * kStageBytes);
-  __shared__ uint64_t full[2], empty[2], tfull[8], tempty[8];
+  unsigned char* ring = sB + (size_t)NT * CP * 2;
+  constexpr int kPiece = 32 * DP * 2;                      // 32 rows of one output block: contiguous in global memory
+  unsigned char* stg = ring + (size_t)S * kAtomBytes;      // two pieces per epilogue warp
+  float* sBias = reinterpret_cast<float*>(stg + (size_t)kEpi2 * 2 * kPiece);
+  __shared__ uint64_t full[8], empty[8], tfull, tempty[8];
   __shared__ uint32_t tmem_s;
   __shared__ int abort_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  for (int i = tid; i < NT * CP * 2 / 16; i += kThreads)
+  for (int i = tid; i < NT * CP * 2 / 16; i += kThreads2)
     reinterpret_cast<uint4*>(sB)[i] = __ldg(reinterpret_cast<const uint4*>(u.Bimg) + i);
-  for (int i = tid; i < NT; i += kThreads) sBias[i] = u.bias ? u.bias[i] : 0.f;
+  for (int i = tid; i < NT; i += kThreads2) sBias[i] = u.bias ? u.bias[i] : 0.f;
   fence_proxy_async();
   if (tid == 0) {
     abort_s = 0;
-    for (int i = 0; i < 2; ++i) { mbar_init(&full[i], kLoadWarps); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 8; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], kEpiWarps); }
+    for (int i = 0; i < 8; ++i) { mbar_init(&full[i], 2); mbar_init(&empty[i], 1); }
+    mbar_init(&tfull, 1);
+    for (int i = 0; i < 8; ++i) mbar_init(&tempty[i], kEpi2);
     mbar_init_fence();
   }
   const uint32_t tcols = pow2_cols(NT);
-  if (warp == kEpiWarps) tmem_alloc(&tmem_s, tcols);
+  if (warp == kEpi2) tmem_alloc(&tmem_s, tcols);
   fence_before_sync();
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem = tmem_s;
   const long long n_tiles = (u.n_windows + 1) / 2;
 
-  if (warp > kEpiWarps) {
-    // ---------------- loaders: warp lw owns window column lw of every window row.  Asynchronous
-    // 8-byte copies land directly in the swizzled operand image; a stage is published one tile
-    // late (after its copies have completed), so two tiles of loads are in flight per SM.
-    const int lw = warp - kEpiWarps - 1;
-    constexpr int NPC = (CP / 4 + 31) / 32;      // 8-byte pieces per lane per row
-    // Per-lane constants: tile row r = lw + 8*(8*half + a) has (r & 7) == lw, so the swizzled
-    // destination of a piece is a fixed offset plus 1024 bytes per row step.
-    uint32_t dst0[NPC];
-    int colb[NPC];                                // byte offset of the piece inside a source row, -1 = padding
-#pragma unroll
-    for (int pi = 0; pi < NPC; ++pi) {
-      const int col = (lane + 32 * pi) * 4;
-      dst0[pi] = (uint32_t)((col >> 6) * kAtomBytesA) + sw128_offset(lw, col & 63);
-      colb[pi] = col < u.kvalid ? col * 2 : -1;
-    }
+  if (warp > kEpi2) {
+    // ---------------- loaders
+    const int set = (warp - kEpi2 - 1) >> 1;
+    LoaderLane ll;
+    ll.init(((warp - kEpi2 - 1) & 1) * 32 + lane);
     const char* const srcA = reinterpret_cast<const char*>(u.A);
-    const long long row_bytes = (long long)u.lda * 2;
+    const long long row_bytes = (long long)u.lda * 2, line_bytes = (long long)u.W * row_bytes;
+    const uint32_t ringA = smem_u32(ring);
+    RingPos rp;
+    rp.init(set, S);
+    int g = set;                                 // ring step = tile iteration * NA + atom
     int it = 0;
     for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
-      const int stage = it & 1;
-      if (!wait_bar_warp(&empty[stage], ((it >> 1) & 1) ^ 1, &abort_s, L.err)) break;
-      const uint32_t sA = smem_u32(sA0 + stage * kStageBytes);
+      // the two windows of the pair: cyclic shift + partition are this address arithmetic
+      const char* col0[2];
+      int i0[2];
+      bool wv[2];
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
-        // one window of the pair: cyclic shift + partition are this address arithmetic
         const int win = 2 * (int)tile + half;
-        const bool wv = win < (int)u.n_windows;
+        wv[half] = win < (int)u.n_windows;
         const int b = win / u.nW, w = win - b * u.nW;
         const int wi = w / u.nWw, wj = w - wi * u.nWw;
-        int j = wj * 8 + lw + u.s;
+        int j = wj * 8 + ll.lw + u.s;
         if (j >= u.W) j -= u.W;
-        const int i0 = wi * 8 + u.s;
-        const char* col0 = srcA + ((long long)b * u.H * u.W + j) * row_bytes;
-        const long long line_bytes = (long long)u.W * row_bytes;
+        i0[half] = wi * 8 + u.s;
+        col0[half] = srcA + ((long long)b * u.H * u.W + j) * row_bytes + ll.pp * 16;
+      }
+      bool ok = true;
+      for (; g < (it + 1) * NA; g += kSets) {
+        const int atom = g - it * NA;
+        if (!wait_bar_warp(&empty[rp.slot], rp.ph ^ 1, &abort_s, L.err)) { ok = false; break; }
+        const uint32_t dst = ringA + rp.slot * kAtomBytes + ll.dst0;
+        const int colb = atom * 128 + ll.pp * 16;          // byte offset inside a source row
+        const bool v0 = colb < u.kvalid * 2, v1 = colb + 8 < u.kvalid * 2;
 #pragma unroll
-        for (int a = 0; a < 8; ++a) {
-          int i = i0 + a;
-          if (i >= u.H) i -= u.H;
-          const char* src = col0 + i * line_bytes;
+        for (int half = 0; half < 2; ++half) {
 #pragma unroll
-          for (int pi = 0; pi < NPC; ++pi) {
-            if ((lane + 32 * pi) * 4 < CP) {
-              const bool v = wv && colb[pi] >= 0;
-              cp_async8(sA + dst0[pi] + (8 * half + a) * 1024, v ? src + colb[pi] : srcA, v);
-            }
+          for (int a8 = 0; a8 < 8; ++a8) {
+            int i = i0[half] + a8;
+            if (i >= u.H) i -= u.H;
+            const char* src = col0[half] + i * line_bytes + atom * 128;
+            const uint32_t d = dst + (8 * half + a8) * 1024;
+            cp_async8(d, wv[half] && v0 ? src : srcA, wv[half] && v0);
+            cp_async8(d + 8, wv[half] && v1 ? src + 8 : srcA, wv[half] && v1);
           }
         }
+        cp_async_commit();
+        cp_async_wait(0);
+        publish(&full[rp.slot], lane);
+        rp.advance(kSets, S);
       }
-      cp_async_commit();
-      if (it > 0) {
-        cp_async_wait(1);
-        publish(&full[(it - 1) & 1], lane);
-      }
+      if (!ok) break;
     }
     cp_async_wait(0);
-    if (it > 0 && __all_sync(0xffffffffu, abort_s == 0)) publish(&full[(it - 1) & 1], lane);
-  } else if (warp == kEpiWarps) {
-    // ---------------- MMA issue
+  } else if (warp == kEpi2) {
+    // ---------------- MMA issue.  Descriptors advance by adding to their address field.  All K atoms
+    // of a tile are consumed accumulator by accumulator (switching the accumulator between
+    // consecutive MMAs costs about as much as two MMAs of this width).
     if (lane == 0) {
       const uint32_t idesc = make_idesc(128, u.cw, 0, 0);
-      const uint32_t bAddr = smem_u32(sB);
+      const uint64_t a0 = make_desc(smem_u32(ring), 16, 1024), b0 = make_desc(smem_u32(sB), 16, 1024);
+      RingPos rp;
+      rp.init(0, S);
       int it = 0;
       bool ok = true;
       for (long long tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
-        const int stage = it & 1;
-        if (!wait_bar(&full[stage], (it >> 1) & 1, &abort_s, L.err)) break;
-        fence_after_sync();
-        const uint32_t aAddr = smem_u32(sA0 + stage * kStageBytes);
-        for (int c = 0; c < u.nchunks; ++c) {
+        int slot_a[NA];
+        for (int c = 0; c < u.nchunks && ok; ++c) {
           if (!wait_bar(&tempty[c], (it & 1) ^ 1, &abort_s, L.err)) { ok = false; break; }
           fence_after_sync();
 #pragma unroll
-          for (int kk = 0; kk < CP / 16; ++kk) {
-            const uint64_t ad = make_desc(aAddr + (kk >> 2) * kAtomBytesA + (kk & 3) * 32, 16, 1024);
-            const uint64_t bd = make_desc(bAddr + (kk >> 2) * (NT * 128) + c * u.cw * 128 + (kk & 3) * 32, 16, 1024);
-            mma_bf16(tmem + c * u.cw, ad, bd, idesc, kk > 0);
+          for (int atom = 0; atom < NA; ++atom) {
+            if (c == 0) {
+              if (!wait_bar(&full[rp.slot], rp.ph, &abort_s, L.err)) { ok = false; break; }
+              fence_after_sync();
+              slot_a[atom] = rp.slot;
+              rp.advance(1, S);
+            }
+            const uint64_t ad = a0 + (uint64_t)((slot_a[atom] * kAtomBytes) >> 4);
+            const uint64_t bd = b0 + (uint64_t)(((atom * NT + c * u.cw) * 128) >> 4);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) mma_bf16(tmem + c * u.cw, ad + 2 * kk, bd + 2 * kk, idesc, (atom | kk) != 0);
           }
-          commit(&tfull[c]);
         }
-        commit(&empty[stage]);
+        if (!ok) break;
+#pragma unroll
+        for (int atom = 0; atom < NA; ++atom) commit(&empty[slot_a[atom]]);
+        commit(&tfull);
       }
     }
   } else {
-    // ---------------- epilogue: thread = accumulator row = (window of the pair, slot)
-    const int r = tid;
+    // ---------------- epilogue: accumulator row = (window of the pair, slot).  A warp owns 32 rows; the
+    // 32 rows of one output block are contiguous in the global tile image, so the warp builds that
+    // piece in its private staging buffer and ships it with one bulk copy (two buffers alternate).
+    const int quad = warp & 3, half = warp >> 2;
+    const int row = (quad & 1) * 32 + lane;       // slot inside the window
     const int nblk = u.cw / DP;
-    int it = 0;
+    unsigned char* mystg = stg + (size_t)warp * 2 * kPiece;
+    const uint32_t mystgA = smem_u32(mystg);
+    int it = 0, nst = 0;
     bool ok = true;
     for (long long tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
-      const long long win = 2 * tile + (r >> 6);
+      const long long win = 2 * tile + (quad >> 1);
       const bool valid = win < u.n_windows;
-      __nv_bfloat16* orow = u.out + win * u.win_stride + (r & 63) * DP;
+      __nv_bfloat16* obase = u.out + win * u.win_stride + (quad & 1) * 32 * DP;
+      if (!wait_bar_warp(&tfull, it & 1, &abort_s, L.err)) break;
+      fence_after_sync();
       for (int c = 0; c < u.nchunks; ++c) {
-        if (!wait_bar_warp(&tfull[c], it & 1, &abort_s, L.err)) { ok = false; break; }
-        fence_after_sync();
         for (int blk = 0; blk < nblk; ++blk) {
+          const int gb = c * nblk + blk;
+          if ((gb & 1) != half) continue;          // the two warps of a quadrant alternate blocks
           uint32_t v[DP];
-          const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + c * u.cw + blk * DP;
+          const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + gb * DP;
           if constexpr (DP == 32) tmem_ld32(taddr, v); else tmem_ld16(taddr, v);
-          tmem_ld_wait();
-          const int gb = c * nblk + blk, n0 = c * u.cw + blk * DP;
-          const float sc = (u.q_every3 && gb % 3 == 0) ? u.qscale : 1.f;
-          uint32_t o[DP / 2];
-#pragma unroll
-          for (int j = 0; j < DP / 2; ++j)
-            o[j] = pack_bf16((__uint_as_float(v[2 * j]) + sBias[n0 + 2 * j]) * sc,
-                             (__uint_as_float(v[2 * j + 1]) + sBias[n0 + 2 * j + 1]) * sc);
-          if (valid) {
-            uint4* dst = reinterpret_cast<uint4*>(orow + (long long)gb * 64 * DP);
-#pragma unroll
-            for (int j = 0; j < DP / 8; ++j) dst[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+          const int buf = nst & 1;
+          if (nst >= 2) {                          // the copy that last read this buffer has finished reading
+            if (lane == 0) bulk_wait_read1();
+            __syncwarp();
           }
+          tmem_ld_wait();
+          const float sc = (u.q_every3 && gb % 3 == 0) ? u.qscale : 1.f;
+          unsigned char* piece = mystg + buf * kPiece - (quad & 1) * kPiece;   // tile_off counts rows from the block start
+#pragma unroll
+          for (int j = 0; j < DP / 8; ++j) {
+            const float4 b0v = *reinterpret_cast<const float4*>(sBias + gb * DP + 8 * j);
+            const float4 b1v = *reinterpret_cast<const float4*>(sBias + gb * DP + 8 * j + 4);
+            uint4 o;
+            o.x = pack_bf16((__uint_as_float(v[8 * j]) + b0v.x) * sc, (__uint_as_float(v[8 * j + 1]) + b0v.y) * sc);
+            o.y = pack_bf16((__uint_as_float(v[8 * j + 2]) + b0v.z) * sc, (__uint_as_float(v[8 * j + 3]) + b0v.w) * sc);
+            o.z = pack_bf16((__uint_as_float(v[8 * j + 4]) + b1v.x) * sc, (__uint_as_float(v[8 * j + 5]) + b1v.y) * sc);
+            o.w = pack_bf16((__uint_as_float(v[8 * j + 6]) + b1v.z) * sc, (__uint_as_float(v[8 * j + 7]) + b1v.w) * sc);
+            *reinterpret_cast<uint4*>(piece + tile_off<DP>(row, j)) = o;
+          }
+          fence_proxy_async();                     // the bulk copy reads these stores through the async proxy
+          __syncwarp();
+          if (lane == 0) {
+            if (valid) bulk_store(obase + (long long)gb * 64 * DP, mystgA + buf * kPiece, kPiece);
+            else bulk_commit();
+          }
+          ++nst;
         }
         fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(&tempty[c]);
       }
     }
+    if (lane == 0) bulk_wait_all();
   }
   fence_before_sync();
   __syncthreads();
-  if (warp == kEpiWarps) {
+  if (warp == kEpi2) {
     __syncwarp();
     tmem_dealloc(tmem, tcols);
   }
@@ -238,111 +341,97 @@ __global__ void __launch_bounds__(kThreads, 1) gw_kernel(const __grid_constant__
 // ==========================================================================================
 // gt_kernel
 // ==========================================================================================
-constexpr int kAtomStage = 128 * 128;   // one K atom of a 128-row tile: 16 KB
 
-__global__ void __launch_bounds__(kThreads, 1) gt_kernel(const __grid_constant__ GTLaunch L) {
+__global__ void __launch_bounds__(kThreads2, 1) gt_kernel(const __grid_constant__ GTLaunch L) {
   const GTSplit& sp = L.s[blockIdx.y];
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = align1024(smem_raw);
   const int NB = L.NB, natoms = L.natoms, S = L.nstages;
   unsigned char* sB = sm;
   unsigned char* ring = sB + (size_t)natoms * NB * 128;
-  unsigned char* stg = ring + (size_t)S * kAtomStage;
+  unsigned char* stg = ring + (size_t)S * kAtomBytes;
   float* sBias = reinterpret_cast<float*>(stg + (size_t)128 * NB * 2);
   __shared__ uint64_t full[8], empty[8], tfull[2], tempty[2];
   __shared__ uint32_t tmem_s;
   __shared__ int abort_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  for (int i = tid; i < natoms * NB * 8; i += kThreads)
+  for (int i = tid; i < natoms * NB * 8; i += kThreads2)
     reinterpret_cast<uint4*>(sB)[i] = __ldg(reinterpret_cast<const uint4*>(sp.Bimg) + i);
-  for (int i = tid; i < NB; i += kThreads) sBias[i] = sp.bias ? sp.bias[i] : 0.f;
+  for (int i = tid; i < NB; i += kThreads2) sBias[i] = sp.bias ? sp.bias[i] : 0.f;
   fence_proxy_async();
   if (tid == 0) {
     abort_s = 0;
-    for (int i = 0; i < 8; ++i) { mbar_init(&full[i], kLoadWarps); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], kEpiWarps); }
+    for (int i = 0; i < 8; ++i) { mbar_init(&full[i], 2); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], kEpi2); }
     mbar_init_fence();
   }
   const uint32_t tcols = pow2_cols(2 * NB);
-  if (warp == kEpiWarps) tmem_alloc(&tmem_s, tcols);
+  if (warp == kEpi2) tmem_alloc(&tmem_s, tcols);
   fence_before_sync();
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem = tmem_s;
   const long long n_tiles = (L.rows + 127) / 128;
 
-  if (warp > kEpiWarps) {
-    // ---------------- loaders: thread -> (8-byte piece of the atom, 8 rows), asynchronous copies;
-    // a ring stage is published `lag` steps after it was issued, once its copies have landed.
-    const int tl = tid - 32 * (kEpiWarps + 1);
-    const int piece = tl & 15, row0 = tl >> 4;
-    const int lag = S - 1 < 3 ? S - 1 : 3;
-    const uint32_t ringA = smem_u32(ring);
-    // rows row0 + 16k share (row & 7), so a piece's swizzled destination is dst0 + 2048 k
-    const uint32_t dst0 = sw128_offset(row0, piece * 4);
+  if (warp > kEpi2) {
+    // ---------------- loaders (four sets of two warps, see above)
+    const int set = (warp - kEpi2 - 1) >> 1;
+    LoaderLane ll;
+    ll.init(((warp - kEpi2 - 1) & 1) * 32 + lane);
     const char* const srcA = reinterpret_cast<const char*>(L.A);
     const long long row_bytes = (long long)L.lda * 2;
-    int st = 0, ph = 0, n = 0, pub = 0;          // pub: ring stage of the oldest unpublished step
-    bool ok = true;
-    for (long long tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-      const long long trow = tile * 128 + row0;
-      const char* const src_t = srcA + trow * row_bytes + piece * 8;
+    const uint32_t ringA = smem_u32(ring);
+    RingPos rp;
+    rp.init(set, S);
+    int g = set, it = 0;
+    for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+      const long long trow = tile * 128 + ll.lw;
+      const char* const src_t = srcA + trow * row_bytes + ll.pp * 16;
       const bool full_tile = (tile + 1) * 128 <= L.rows;
-      for (int atom = 0; atom < natoms; ++atom) {
-        if (!wait_bar_warp(&empty[st], ph ^ 1, &abort_s, L.err)) { ok = false; break; }
-        const bool cv = atom * 64 + piece * 4 < L.kvalid;
-        const uint32_t sA = ringA + st * kAtomStage + dst0;
+      bool ok = true;
+      for (; g < (it + 1) * natoms; g += kSets) {
+        const int atom = g - it * natoms;
+        if (!wait_bar_warp(&empty[rp.slot], rp.ph ^ 1, &abort_s, L.err)) { ok = false; break; }
+        const uint32_t dst = ringA + rp.slot * kAtomBytes + ll.dst0;
+        const int colb = atom * 128 + ll.pp * 16;
+        const bool v0 = colb < L.kvalid * 2, v1 = colb + 8 < L.kvalid * 2;
         const char* src = src_t + atom * 128;
-        if (full_tile) {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) cp_async8(sA + k * 2048, cv ? src + k * 16 * row_bytes : srcA, cv);
-        } else {
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const bool v = cv && trow + 16 * k < L.rows;
-            cp_async8(sA + k * 2048, v ? src + k * 16 * row_bytes : srcA, v);
-          }
+        for (int k = 0; k < 16; ++k) {
+          const bool rv = full_tile || trow + 8 * k < L.rows;
+          cp_async8(dst + k * 1024, rv && v0 ? src + k * 8 * row_bytes : srcA, rv && v0);
+          cp_async8(dst + k * 1024 + 8, rv && v1 ? src + k * 8 * row_bytes + 8 : srcA, rv && v1);
         }
         cp_async_commit();
-        if (++st == S) { st = 0; ph ^= 1; }
-        if (++n > lag) {
-          cp_async_wait(lag);
-          publish(&full[pub], lane);
-          if (++pub == S) pub = 0;
-        }
+        cp_async_wait(0);
+        publish(&full[rp.slot], lane);
+        rp.advance(kSets, S);
       }
+      if (!ok) break;
     }
-    {
-      int left = n < lag ? n : lag;              // steps issued but not yet published
-      while (left > 0) {
-        cp_async_wait(left - 1);
-        if (ok) publish(&full[pub], lane);
-        if (++pub == S) pub = 0;
-        --left;
-      }
-    }
-  } else if (warp == kEpiWarps) {
+    cp_async_wait(0);
+  } else if (warp == kEpi2) {
     if (lane == 0) {
       const uint32_t idesc = make_idesc(128, NB, 0, 0);
-      const uint32_t bAddr = smem_u32(sB), rAddr = smem_u32(ring);
-      int st = 0, ph = 0, it = 0;
+      const uint64_t a0 = make_desc(smem_u32(ring), 16, 1024), b0 = make_desc(smem_u32(sB), 16, 1024);
+      RingPos rp;
+      rp.init(0, S);
+      int it = 0;
       bool ok = true;
       for (long long tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
         const int buf = it & 1;
         if (!wait_bar(&tempty[buf], ((it >> 1) & 1) ^ 1, &abort_s, L.err)) break;
         fence_after_sync();
         for (int atom = 0; atom < natoms; ++atom) {
-          if (!wait_bar(&full[st], ph, &abort_s, L.err)) { ok = false; break; }
+          if (!wait_bar(&full[rp.slot], rp.ph, &abort_s, L.err)) { ok = false; break; }
           fence_after_sync();
+          const uint64_t ad = a0 + (uint64_t)((rp.slot * kAtomBytes) >> 4);
+          const uint64_t bd = b0 + (uint64_t)((atom * NB * 128) >> 4);
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {
-            const uint64_t ad = make_desc(rAddr + st * kAtomStage + kk * 32, 16, 1024);
-            const uint64_t bd = make_desc(bAddr + atom * (NB * 128) + kk * 32, 16, 1024);
-            mma_bf16(tmem + buf * NB, ad, bd, idesc, (atom | kk) != 0);
-          }
-          commit(&empty[st]);
-          if (++st == S) { st = 0; ph ^= 1; }
+          for (int kk = 0; kk < 4; ++kk) mma_bf16(tmem + buf * NB, ad + 2 * kk, bd + 2 * kk, idesc, (atom | kk) != 0);
+          commit(&empty[rp.slot]);
+          rp.advance(1, S);
         }
         if (ok) commit(&tfull[buf]);
       }
@@ -350,50 +439,54 @@ __global__ void __launch_bounds__(kThreads, 1) gt_kernel(const __grid_constant__
   } else {
     // ---------------- epilogue: stage the warp's 32 rows in shared memory, then store row pieces
     const int ncols = sp.ncols, n8 = ncols / 4;
-    unsigned char* mystg = stg + (size_t)warp * 32 * ncols * 2;
+    const int quad = warp & 3, half = warp >> 2;
+    unsigned char* mystg = stg + (size_t)quad * 32 * ncols * 2;
     int it = 0;
     for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
       const int buf = it & 1;
-      if (!wait_bar_warp(&tfull[buf], (it >> 1) & 1, &abort_s, L.err)) break;
+      // the vote is also the barrier after which last tile's staging rows may be overwritten
+      if (!pair_vote(quad, wait_bar_warp(&tfull[buf], (it >> 1) & 1, &abort_s, L.err))) break;
       fence_after_sync();
-      for (int c0 = 0; c0 < ncols; c0 += 32) {
+      for (int c0 = 32 * half; c0 < ncols; c0 += 64) {   // the two warps of a quadrant alternate column chunks
         uint32_t v[32];
-        tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + buf * NB + c0, v);
+        tmem_ld32(tmem + ((uint32_t)(quad * 32) << 16) + buf * NB + c0, v);
         tmem_ld_wait();
         // the lane's row of the staging tile; rows are 2*ncols bytes apart (a multiple of 8, and an
         // odd multiple for C = 180, so these 8-byte stores do not collide on banks)
         uint2* dst = reinterpret_cast<uint2*>(mystg + ((size_t)lane * ncols + c0) * 2);
 #pragma unroll
         for (int j = 0; j < 8; ++j)
-          if (c0 + 4 * j < ncols)
-            dst[j] = make_uint2(pack_bf16(__uint_as_float(v[4 * j]) + sBias[c0 + 4 * j],
-                                          __uint_as_float(v[4 * j + 1]) + sBias[c0 + 4 * j + 1]),
-                                pack_bf16(__uint_as_float(v[4 * j + 2]) + sBias[c0 + 4 * j + 2],
-                                          __uint_as_float(v[4 * j + 3]) + sBias[c0 + 4 * j + 3]));
+          if (c0 + 4 * j < ncols) {
+            const float4 bq = *reinterpret_cast<const float4*>(sBias + c0 + 4 * j);
+            dst[j] = make_uint2(pack_bf16(__uint_as_float(v[4 * j]) + bq.x, __uint_as_float(v[4 * j + 1]) + bq.y),
+                                pack_bf16(__uint_as_float(v[4 * j + 2]) + bq.z, __uint_as_float(v[4 * j + 3]) + bq.w));
+          }
       }
       fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tempty[buf]);
-      // copy-out: lane = 8-byte piece of a row (two pieces per lane cover up to 256 columns)
-      const long long trow0 = tile * 128 + warp * 32;
+      pair_sync(quad);                           // both halves of the staging rows are written
+      // copy-out: lane = 8-byte piece of a row (two pieces per lane cover up to 256 columns); each
+      // warp of the pair stores 16 of the quadrant's 32 rows
+      const long long trow0 = tile * 128 + quad * 32;
       const int nrows = L.rows - trow0 < 32 ? (int)(L.rows - trow0) : 32;
       char* const obase = reinterpret_cast<char*>(L.out + trow0 * L.ldo + sp.col0) + lane * 8;
       const long long obytes = (long long)L.ldo * 2;
       const unsigned char* sbase = mystg + lane * 8;
       const bool p0 = lane < n8, p1 = lane + 32 < n8;
+      const int rend = nrows < 16 * half + 16 ? nrows : 16 * half + 16;
 #pragma unroll 4
-      for (int rr = 0; rr < nrows; ++rr) {
+      for (int rr = 16 * half; rr < rend; ++rr) {
         if (p0) *reinterpret_cast<uint2*>(obase + rr * obytes) = *reinterpret_cast<const uint2*>(sbase + rr * ncols * 2);
         if (p1)
           *reinterpret_cast<uint2*>(obase + rr * obytes + 256) =
               *reinterpret_cast<const uint2*>(sbase + rr * ncols * 2 + 256);
       }
-      __syncwarp();
     }
   }
   fence_before_sync();
   __syncthreads();
-  if (warp == kEpiWarps) {
+  if (warp == kEpi2) {
     __syncwarp();
     tmem_dealloc(tmem, tcols);
   }
@@ -637,13 +730,19 @@ static int launch_gw_t(const GWLaunch& L, int nunits, cudaStream_t st, const cha
     const long long t = (L.u[i].n_windows + 1) / 2;
     if (t > max_tiles) max_tiles = t;
   }
-  const size_t smem = 1024 + (size_t)maxNT * CP * 2 + 2 * 128 * CP * 2 + (size_t)maxNT * 4 + 64;
+  const size_t fixed = 1024 + (size_t)maxNT * CP * 2 + (size_t)kEpi2 * 2 * 32 * DP * 2 + (size_t)maxNT * 4 + 64;
+  int nslots = (int)((215 * 1024 - fixed) / (128 * 128));
+  if (nslots > 8) nslots = 8;
+  if (nslots < CP / 64 + 1 || nslots < 4) return GSWA_ERR_UNSUPPORTED;
+  const size_t smem = fixed + (size_t)nslots * 128 * 128;
   if (cudaFuncSetAttribute(gw_kernel<CP, DP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return check_launch();
+  GWLaunch Lc = L;
+  Lc.nslots = nslots;
   long long gx = num_sms() / nunits;
   if (gx < 1) gx = 1;
   if (gx > max_tiles) gx = max_tiles;
-  { KernelScope ks_(name, st); gw_kernel<CP, DP><<<dim3((unsigned)gx, nunits), kThreads, smem, st>>>(L); }
+  { KernelScope ks_(name, st); gw_kernel<CP, DP><<<dim3((unsigned)gx, nunits), kThreads2, smem, st>>>(Lc); }
   return check_launch();
 }
 
@@ -656,7 +755,7 @@ int launch_gw(const GWLaunch& L, int nunits, int Cp, int dp, cudaStream_t st, co
 }
 
 size_t gt_smem_bytes(int natoms, int NB, int nstages) {
-  return 1024 + (size_t)natoms * NB * 128 + (size_t)nstages * kAtomStage + (size_t)128 * NB * 2 + (size_t)NB * 4 + 64;
+  return 1024 + (size_t)natoms * NB * 128 + (size_t)nstages * kAtomBytes + (size_t)128 * NB * 2 + (size_t)NB * 4 + 64;
 }
 
 int launch_gt(const GTLaunch& L, int nsplits, cudaStream_t st, const char* name) {
@@ -667,7 +766,7 @@ int launch_gt(const GTLaunch& L, int nsplits, cudaStream_t st, const char* name)
   long long gx = num_sms() / nsplits;
   if (gx < 1) gx = 1;
   if (gx > n_tiles) gx = n_tiles;
-  { KernelScope ks_(name, st); gt_kernel<<<dim3((unsigned)gx, nsplits), kThreads, smem, st>>>(L); }
+  { KernelScope ks_(name, st); gt_kernel<<<dim3((unsigned)gx, nsplits), kThreads2, smem, st>>>(L); }
   return check_launch();
 }
 
