@@ -89,6 +89,27 @@ int gswa_forward(const gswa_desc* desc, const void* x, const void* w_qkv, const 
                  const void* b_proj, const void* bias_table, void* y, void* saved, void* scratch,
                  size_t scratch_bytes, void* cuda_stream);
 
+/* Inference forward for callers that cannot allocate device memory (the paper has no counterpart).
+ * Some hosts hand a library its input and output buffers and nothing else: a plug-in loaded into an
+ * application that owns all device memory, a C program without an allocator for the GPU, a real-time
+ * loop in which cudaMalloc (which may synchronise the whole device) is not acceptable.  gswa_forward
+ * needs `infer_scratch_bytes` of scratch from such a caller; this variant takes none.  It computes
+ * exactly what gswa_forward computes with saved == NULL, and keeps its intermediates (projected q,k,v
+ * tiles, attention output, weight images) in one array that is part of the library's device image:
+ * GSWA_STATIC_SCRATCH_BYTES bytes, held on every GPU that loads the library until the process exits.
+ *   - A layer whose infer_scratch_bytes (gswa_workspace_query) exceeds GSWA_STATIC_SCRATCH_BYTES is
+ *     rejected with GSWA_ERR_WORKSPACE before anything is enqueued; nothing is ever allocated or freed,
+ *     by this call or by anything it calls.
+ *   - The first call on a device looks the array's device address up (once per device, with the
+ *     caller's current device); make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the last call's contents; what has to
+ *     start from zero is cleared by each call.  Two calls whose work overlaps on the GPU (different
+ *     streams, or different threads) race on it: serialise them.
+ * x, the parameters and y are the caller's device buffers as for gswa_forward. */
+#define GSWA_STATIC_SCRATCH_BYTES (16u << 20)
+int gswa_forward_static(const gswa_desc* desc, const void* x, const void* w_qkv, const void* b_qkv,
+                        const void* w_proj, const void* b_proj, const void* bias_table, void* y, void* cuda_stream);
+
 /* Backward pass (reverse mode of gswa_forward; the paper's stated target is the memory of
  * back-propagation).  `saved` is the buffer written by gswa_forward for the same desc and inputs.
  * Writes dx (element type `dtype`) and the float32 parameter gradients dw_qkv[3C,C], db_qkv[3C],

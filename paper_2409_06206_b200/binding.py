@@ -17,7 +17,9 @@ LIB_PATH = os.path.join(_PKG, "libgswa.so")
 GSWA_F32, GSWA_BF16 = 0, 1
 FLAG_ACCUMULATE, FLAG_GENERIC = 1, 2
 
-EXPORTS = ("gswa_workspace_query", "gswa_forward", "gswa_backward", "gswa_index_maps", "gswa_step_host",
+STATIC_SCRATCH_BYTES = 16 << 20
+
+EXPORTS = ("gswa_workspace_query", "gswa_forward", "gswa_forward_static", "gswa_backward", "gswa_index_maps", "gswa_step_host",
            "gswa_scratch_status", "gswa_profile_enable", "gswa_profile_read", "gswa_launch_count", "gswa_status_string")
 
 
@@ -79,6 +81,8 @@ def lib() -> C.CDLL:
         szp = C.POINTER(C.c_size_t)
         L.gswa_workspace_query.argtypes = [dp, szp, szp, szp, szp]
         L.gswa_forward.argtypes = [dp] + [vp] * 9 + [sz, vp]
+        L.gswa_forward_static.argtypes = [dp] + [vp] * 8
+        L.gswa_forward_static.restype = C.c_int
         L.gswa_backward.argtypes = [dp] + [vp] * 14 + [sz, vp]
         L.gswa_index_maps.argtypes = [dp, C.c_int32] + [vp] * 6
         L.gswa_step_host.argtypes = [dp] + [vp] * 15 + [sz, szp, vp]
@@ -137,6 +141,15 @@ def gswa_forward(desc: Desc, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, y, sav
         scratch_bytes = 0 if scratch is None else scratch.numel() * scratch.element_size()
     _check(lib().gswa_forward(C.byref(desc.c), _ptr(x), _ptr(w_qkv), _ptr(b_qkv), _ptr(w_proj), _ptr(b_proj),
                               _ptr(bias_table), _ptr(y), _ptr(saved), _ptr(scratch), scratch_bytes, _stream(stream)))
+
+
+def gswa_forward_static(desc: Desc, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, y, stream=None) -> None:
+    """Inference forward without any caller-provided scratch: for hosts that cannot allocate device memory.
+
+    The library keeps the intermediates in a fixed array of STATIC_SCRATCH_BYTES inside its own device image;
+    larger layers raise GswaError(-5).  Calls share that array, so calls that overlap on the GPU race."""
+    _check(lib().gswa_forward_static(C.byref(desc.c), _ptr(x), _ptr(w_qkv), _ptr(b_qkv), _ptr(w_proj), _ptr(b_proj),
+                                     _ptr(bias_table), _ptr(y), _stream(stream)))
 
 
 def gswa_backward(desc: Desc, x, w_qkv, b_qkv, w_proj, bias_table, saved, dy, dx, dw_qkv, db_qkv, dw_proj, db_proj,

@@ -101,6 +101,32 @@ int make_plan(const gswa_desc* desc, Plan* p) {
 
 static bool misaligned(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) != 0; }
 
+// Scratch of gswa_forward_static: part of the device image, so no allocation call is ever made for
+// it.  In host code this name is only a handle; the device address is looked up per device below.
+static __device__ __align__(256) unsigned char g_static_scratch[GSWA_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_static_mu;
+static void* g_static_ptr[kMaxDevices] = {};
+
+// Device address of g_static_scratch on the current device (looked up once per device).
+static int static_scratch(void** out) {
+  int dev = -1;
+  int rc = cuda_rc(cudaGetDevice(&dev));
+  if (rc) return rc;
+  if (dev < 0 || dev >= kMaxDevices) return GSWA_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lk(g_static_mu);
+  if (g_static_ptr[dev] == nullptr) {
+    void* ptr = nullptr;
+    rc = cuda_rc(cudaGetSymbolAddress(&ptr, g_static_scratch));
+    if (rc) return rc;
+    if (ptr == nullptr) return GSWA_ERR_CUDA;
+    g_static_ptr[dev] = ptr;
+  }
+  *out = g_static_ptr[dev];
+  return GSWA_OK;
+}
+
 }  // namespace gswa
 
 using namespace gswa;
@@ -141,6 +167,20 @@ int gswa_forward(const gswa_desc* desc, const void* x, const void* w_qkv, const 
   }
   void* carry = saved ? saved : scratch;
   return generic_forward(p, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, y, carry, st);
+}
+
+int gswa_forward_static(const gswa_desc* desc, const void* x, const void* w_qkv, const void* b_qkv,
+                        const void* w_proj, const void* b_proj, const void* bias_table, void* y, void* cuda_stream) {
+  Plan p;
+  int rc = make_plan(desc, &p);
+  if (rc) return rc;
+  if (p.infer_scratch > (size_t)GSWA_STATIC_SCRATCH_BYTES) return GSWA_ERR_WORKSPACE;   // layer too large for the built-in array
+  void* scratch = nullptr;
+  if ((rc = static_scratch(&scratch))) return rc;
+  // same path as gswa_forward with saved == NULL; the device error word at the head of the scratch
+  // is cleared by that path on every call
+  return gswa_forward(desc, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, y, nullptr, scratch,
+                      (size_t)GSWA_STATIC_SCRATCH_BYTES, cuda_stream);
 }
 
 int gswa_backward(const gswa_desc* desc, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
@@ -291,7 +331,7 @@ const char* gswa_status_string(int status) {
     case GSWA_ERR_SHAPE: return "inconsistent layer description";
     case GSWA_ERR_ALIGN: return "device pointer not 16-byte aligned";
     case GSWA_ERR_UNSUPPORTED: return "layer description not supported";
-    case GSWA_ERR_WORKSPACE: return "scratch or arena buffer too small";
+    case GSWA_ERR_WORKSPACE: return "scratch, arena or built-in scratch array too small for this layer";
     case GSWA_ERR_CUDA: return g_cuda_msg;
     case GSWA_ERR_DEVICE: return "a kernel gave up waiting on an internal barrier; results are invalid";
     default: return "unknown status";
