@@ -49,8 +49,8 @@ int make_units(const Plan& p, Unit* units) {
 
 // Split of the output columns of a token GEMM with K = kvalid so that the resident weight image,
 // the staging tile and at least three ring stages fit.
-bool token_split(int C, int kvalid, TokenSplit* ts) {
-  const int natoms = (kvalid + 63) / 64;
+bool token_split(int C, int K, TokenSplit* ts) {
+  const int natoms = (K + 63) / 64;
   for (int nsplit = 1; nsplit <= kMaxUnits; nsplit *= 2) {
     const int NB = (int)align_up((size_t)(C + nsplit - 1) / nsplit, 32);
     if (NB > 256) continue;
@@ -107,7 +107,7 @@ BwdScratch bwd_layout(const Plan& p, const Unit* units, int nu, const TokenSplit
   BwdScratch s{};
   size_t off = 256;
   s.dO = off; off += align_up((size_t)p.T * p.nh * p.dp * 2, 256);
-  s.dqkv = off; off += align_up((size_t)p.T * 3 * p.C * 2, 256);
+  s.dqkv = off; off += align_up((size_t)p.T * 3 * p.Ap * 2, 256);
   for (int i = 0; i < nu; ++i) {
     s.img[i] = off; off += align_up((size_t)units[i].nheads * p.dp * p.Cp * 2, 256);
   }
@@ -126,29 +126,32 @@ int np_cols(int C) { return (int)align_up((size_t)C + 1, 64); }
 bool fast_path_ok(const Plan& p) {
   if (p.dtype != GSWA_BF16 || (p.flags & GSWA_FLAG_GENERIC)) return false;
   if (p.M != 8 || p.d > 32 || (p.d & 1) || (p.C & 3) || p.C > 252 || p.G > 4) return false;
+  if (p.nh * (p.d <= 16 ? 16 : 32) < 64) return false;       // padded rows must fill one TMA box of 64 columns
   if (p.T >= (1LL << 30) / 4) return false;
   Plan q = p;
   q.dp = p.d <= 16 ? 16 : 32;
   q.Cp = (int)align_up((size_t)p.C, 64);
+  q.Ap = p.nh * q.dp;
   Unit units[kMaxUnits];
   if (make_units(q, units) <= 0) return false;
   TokenSplit a, b;
-  return token_split(p.C, p.C, &a) && token_split(p.C, 3 * p.C, &b);
+  return token_split(p.C, q.Ap, &a) && token_split(p.C, 3 * q.Ap, &b);
 }
 
 void fast_plan_sizes(Plan* p) {
   p->fast = 1;
   p->dp = p->d <= 16 ? 16 : 32;
   p->Cp = (int)align_up((size_t)p->C, 64);
+  p->Ap = p->nh * p->dp;
   Unit units[kMaxUnits];
   const int nu = make_units(*p, units);
   TokenSplit tp, tx;
-  token_split(p->C, p->C, &tp);
-  token_split(p->C, 3 * p->C, &tx);
+  token_split(p->C, p->Ap, &tp);
+  token_split(p->C, 3 * p->Ap, &tx);
   const size_t T = (size_t)p->T;
   p->off_qkv = 0;
   p->off_A = align_up(T * 3 * p->nh * p->dp * 2, 256);
-  p->off_L = p->off_A + align_up(T * p->C * 2, 256);
+  p->off_L = p->off_A + align_up(T * p->Ap * 2, 256);
   p->saved_bytes = p->off_L + align_up(T * p->nh * 4, 256);
   p->fwd_scratch = fwd_layout(*p, units, nu, tp).total;
   p->infer_scratch = p->fwd_scratch + p->saved_bytes;
@@ -179,7 +182,7 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
   Unit units[kMaxUnits];
   const int nu = make_units(p, units);
   TokenSplit tp;
-  if (nu <= 0 || !token_split(p.C, p.C, &tp)) return GSWA_ERR_UNSUPPORTED;
+  if (nu <= 0 || !token_split(p.C, p.Ap, &tp)) return GSWA_ERR_UNSUPPORTED;
   const FwdScratch fs = fwd_layout(p, units, nu, tp);
   const FastGeom geo = make_geom(p);
   char* sc = static_cast<char*>(scratch);
@@ -195,10 +198,10 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
   for (int i = 0; i < nu; ++i)
     jobs[nj++] = PrepJob{PREP_QKV, (const bf*)w_qkv, (const bf*)b_qkv, (unsigned char*)sc + fs.img[i],
                          (float*)(sc + fs.bias[i]), p.C, p.d, p.dp, units[i].h0, units[i].nheads, 0,
-                         units[i].nheads * 3 * p.dp, p.Cp};
+                         units[i].nheads * 3 * p.dp, p.Cp, p.Ap};
   for (int i = 0; i < tp.nsplit; ++i)
     jobs[nj++] = PrepJob{PREP_PROJ, (const bf*)w_proj, (const bf*)b_proj, (unsigned char*)sc + fs.pimg[i],
-                         (float*)(sc + fs.pbias[i]), p.C, p.d, p.dp, 0, 0, i * tp.NB, tp.NB, tp.natoms * 64};
+                         (float*)(sc + fs.pbias[i]), p.C, p.d, p.dp, 0, 0, i * tp.NB, tp.NB, tp.natoms * 64, p.Ap};
   int rc = launch_prep(jobs, nj, st);
   if (rc) return rc;
 
@@ -225,7 +228,8 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
   if ((rc = launch_attn_fwd(al, st))) return rc;
 
   GTLaunch gt{};
-  gt.A = A; gt.lda = p.C; gt.kvalid = p.C; gt.natoms = tp.natoms; gt.rows = p.T;
+  if ((rc = make_tmap(&gt.tmA, A, p.T, p.Ap, 128))) return rc;
+  gt.natoms = tp.natoms; gt.rows = p.T;
   gt.out = (bf*)y; gt.ldo = p.C; gt.NB = tp.NB; gt.nstages = tp.nstages; gt.err = err;
   for (int i = 0; i < tp.nsplit; ++i) {
     const int col0 = i * tp.NB;
@@ -242,7 +246,7 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
   Unit units[kMaxUnits];
   const int nu = make_units(p, units);
   TokenSplit tx;
-  if (nu <= 0 || !token_split(p.C, 3 * p.C, &tx)) return GSWA_ERR_UNSUPPORTED;
+  if (nu <= 0 || !token_split(p.C, 3 * p.Ap, &tx)) return GSWA_ERR_UNSUPPORTED;
   const BwdScratch bs = bwd_layout(p, units, nu, tx);
   const FastGeom geo = make_geom(p);
   char* sc = static_cast<char*>(scratch);
@@ -260,10 +264,10 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
   int nj = 0;
   for (int i = 0; i < nu; ++i)
     jobs[nj++] = PrepJob{PREP_PROJ_T, (const bf*)w_proj, nullptr, (unsigned char*)sc + bs.img[i], nullptr, p.C, p.d,
-                         p.dp, units[i].h0, units[i].nheads, 0, units[i].nheads * p.dp, p.Cp};
+                         p.dp, units[i].h0, units[i].nheads, 0, units[i].nheads * p.dp, p.Cp, p.Ap};
   for (int i = 0; i < tx.nsplit; ++i)
     jobs[nj++] = PrepJob{PREP_QKV_T, (const bf*)w_qkv, nullptr, (unsigned char*)sc + bs.ximg[i], nullptr, p.C, p.d,
-                         p.dp, 0, 0, i * tx.NB, tx.NB, tx.natoms * 64};
+                         p.dp, 0, 0, i * tx.NB, tx.NB, tx.natoms * 64, p.Ap};
   int rc = launch_prep(jobs, nj, st);
   if (rc) return rc;
 
@@ -285,14 +289,19 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
 
   const int sms = 148;
   if (dw_proj || db_proj) {
+    // dW^P = dy^T A (A fetched by TMA); db^P rides on the ones column of A when the head dim is padded
     GRLaunch gr{};
-    gr.L = (const bf*)dy; gr.ldl = p.C; gr.mvalid = p.C;
-    gr.R = A; gr.ldr = p.C; gr.nvalid = p.C; gr.rows = p.T; gr.NP = np_cols(p.C);
+    if ((rc = make_tmap(&gr.tm, A, p.T, p.Ap, 64))) return rc;
+    gr.tma_is_L = 0; gr.use_tma = 1; gr.Q = A; gr.qcols = p.Ap;
+    gr.P = (const bf*)dy; gr.ldp = p.C; gr.pvalid = p.C;
+    gr.Ap = p.Ap; gr.dp = p.dp; gr.d = p.d; gr.C = p.C; gr.M = p.C; gr.rows = p.T;
+    gr.NP = (int)align_up((size_t)p.Ap, 64);
     const int mblocks = (p.C + 127) / 128;
     long long ns = sms / mblocks, cap = (p.T + 63) / 64;
     gr.nsplit = (int)(ns < cap ? (ns < 1 ? 1 : ns) : cap);
-    gr.out = dw_proj ? dw_proj : dummy; gr.colsum = db_proj; gr.err = err;
+    gr.out = dw_proj ? dw_proj : dummy; gr.colsum = p.d < p.dp ? db_proj : nullptr; gr.err = err;
     if ((rc = launch_gr(gr, st, "dwproj_gemm"))) return rc;
+    if (db_proj && p.d == p.dp && (rc = launch_colsum_bf16((const bf*)dy, p.T, p.C, p.C, db_proj, st))) return rc;
   }
 
   AttnLaunch al{};
@@ -303,7 +312,8 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
 
   if (dx) {
     GTLaunch gt{};
-    gt.A = dqkv; gt.lda = 3 * p.C; gt.kvalid = 3 * p.C; gt.natoms = tx.natoms; gt.rows = p.T;
+    if ((rc = make_tmap(&gt.tmA, dqkv, p.T, 3 * p.Ap, 128))) return rc;
+    gt.natoms = tx.natoms; gt.rows = p.T;
     gt.out = (bf*)dx; gt.ldo = p.C; gt.NB = tx.NB; gt.nstages = tx.nstages; gt.err = err;
     for (int i = 0; i < tx.nsplit; ++i) {
       const int col0 = i * tx.NB;
@@ -312,10 +322,14 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
     if ((rc = launch_gt(gt, tx.nsplit, st, "dx_gemm"))) return rc;
   }
   if (dw_qkv || db_qkv) {
+    // dW_qkv = dqkv^T x (dqkv fetched by TMA); db_qkv from a column of ones appended to x
     GRLaunch gr{};
-    gr.L = dqkv; gr.ldl = 3 * p.C; gr.mvalid = 3 * p.C;
-    gr.R = (const bf*)x; gr.ldr = p.C; gr.nvalid = p.C; gr.rows = p.T; gr.NP = np_cols(p.C);
-    const int mblocks = (3 * p.C + 127) / 128;
+    if ((rc = make_tmap(&gr.tm, dqkv, p.T, 3 * p.Ap, 64))) return rc;
+    gr.tma_is_L = 1; gr.use_tma = 1; gr.Q = dqkv; gr.qcols = 3 * p.Ap;
+    gr.P = (const bf*)x; gr.ldp = p.C; gr.pvalid = p.C;
+    gr.Ap = p.Ap; gr.dp = p.dp; gr.d = p.d; gr.C = p.C; gr.M = 3 * p.Ap; gr.rows = p.T;
+    gr.NP = np_cols(p.C);
+    const int mblocks = (3 * p.Ap + 127) / 128;
     long long ns = sms / mblocks, cap = (p.T + 63) / 64;
     gr.nsplit = (int)(ns < cap ? (ns < 1 ? 1 : ns) : cap);
     gr.out = dw_qkv ? dw_qkv : dummy; gr.colsum = db_qkv; gr.err = err;

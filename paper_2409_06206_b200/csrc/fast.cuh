@@ -12,9 +12,16 @@
 // is at the same time the shared-memory image the attention kernels read with ldmatrix: the GEMM
 // epilogue builds the image in shared memory and ships it with one bulk copy, the attention kernels
 // fetch it with plain linear copies.
-// "Token-major" buffers are packed [T, cols] rows in original token order (attention output A[T,C],
-// dqkv[T,3C]); the attention epilogues undo partition and shift when they store into them.
+// "Token-major" buffers hold rows in original token order with the head dim padded like the tiles:
+// attention output A[T, Ap], Ap = heads * DP, and dqkv[T, 3*Ap] (q | k | v, head-major inside each);
+// the attention epilogues undo partition and shift when they store into them.  Their row pitches are
+// multiples of 16 bytes, so the GEMMs that consume them fetch 64-column x 128-row (or 64-row) boxes
+// with TMA, which also applies the 128-byte swizzle the tensor core expects.  Pad columns hold zeros,
+// except A[:, d] of head 0 (when d < DP), which holds ones: multiplied with dy it yields the bias
+// gradient of the output projection for free.
 #pragma once
+
+#include <cuda.h>
 
 #include "gswa_internal.h"
 
@@ -59,15 +66,15 @@ struct GWLaunch {
   int nslots;                  // ring slots of 16 KB (set by launch_gw)
 };
 
-// ---- token GEMM: rows in token order from packed [T, lda], output packed rows [T, ldo]
+// ---- token GEMM: A rows in token order, fetched by TMA from a padded [rows, K] buffer; packed rows out
 struct GTSplit {
   const unsigned char* Bimg;   // [KP/64 atoms][NB rows][128 B]
   const float* bias;           // [NB] or nullptr
   int col0, ncols;             // output columns [col0, col0+ncols) of each row
 };
 struct GTLaunch {
-  const __nv_bfloat16* A;
-  int lda, kvalid, natoms;     // natoms = KP/64
+  CUtensorMap tmA;             // [rows, K] bf16, box 64 columns x 128 rows, 128-byte swizzle
+  int natoms;                  // K atoms of 64 columns
   long long rows;
   __nv_bfloat16* out;
   int ldo;
@@ -77,23 +84,35 @@ struct GTLaunch {
   int* err;
 };
 
-// ---- reduction GEMM: out[m, n] += sum_t L[t, m] R[t, n], plus column sums of L via a ones column
+// ---- reduction GEMM: out[m, n] += sum_t L[t, m] R[t, n].  One operand is a padded token-major buffer
+// fetched by TMA (box 64 columns x 64 rows), the other a packed caller tensor fetched by 8-byte copies.
+//   tma_is_L = 1 (dW_qkv): L = dqkv[T, 3*Ap], R = x[T, C] plus a column of ones at index C
+//   tma_is_L = 0 (dW_proj): L = dy[T, C],      R = A[T, Ap] (whose column d holds ones when d < DP)
+// Padded indices (kind, head, c) map to kind*C + head*d + c; c >= d is dropped.
 struct GRLaunch {
-  const __nv_bfloat16* L;      // [rows, ldl], mvalid valid columns
-  int ldl, mvalid;
-  const __nv_bfloat16* R;      // [rows, ldr], nvalid valid columns
-  int ldr, nvalid;
+  CUtensorMap tm;
+  int use_tma;                 // 1: padded operand through TMA; 0: through 16-byte asynchronous copies
+  const __nv_bfloat16* Q;      // the padded operand [rows, qcols]
+  int qcols;
+  int tma_is_L;
+  const __nv_bfloat16* P;      // the copy-fed operand, [rows, ldp] with pvalid valid columns
+  int ldp, pvalid;
+  int Ap, dp, d, C;
+  int M;                       // extent of the M index space (3*Ap or C)
   long long rows;
-  int NP;                      // padded N (multiple of 64, > nvalid so that column nvalid can carry ones)
+  int NP;                      // accumulator columns (multiple of 64)
   int nsplit;                  // token splits
-  float* out;                  // [mvalid, nvalid] float, accumulated with atomics
-  float* colsum;               // [mvalid] or nullptr: sum_t L[t, m]
+  int nstages;                 // ring depth (set by launch_gr)
+  float* out;                  // float, accumulated with atomics: [3C, C] or [C, C]
+  float* colsum;               // or nullptr: dB[m] = sum_t L[t, m]
   int* err;
 };
 
 int launch_gw(const GWLaunch& L, int nunits, int Cp, int dp, cudaStream_t st, const char* name);
 int launch_gt(const GTLaunch& L, int nsplits, cudaStream_t st, const char* name);
 int launch_gr(const GRLaunch& L, cudaStream_t st, const char* name);
+// Tensor map of a padded token-major bf16 buffer [rows, cols]: box 64 columns x box_rows rows, 128-byte swizzle.
+int make_tmap(CUtensorMap* tm, const void* base, long long rows, int cols, int box_rows);
 
 // Weight images (shared-memory images of the B operands, built once per call by a small kernel).
 enum PrepMode { PREP_QKV = 0, PREP_PROJ_T = 1, PREP_PROJ = 2, PREP_QKV_T = 3 };
@@ -105,6 +124,7 @@ struct PrepJob {
   float* bias_out;             // or nullptr
   int C, d, dp, h0, nheads;    // head range for the per-head modes
   int n0, NT, KP;              // first output row (PREP_PROJ / PREP_QKV_T), rows, padded K
+  int Ap;                      // heads * dp: K of PREP_PROJ / PREP_QKV_T runs over padded (kind, head, c) indices
 };
 int launch_prep(const PrepJob* jobs, int njobs, cudaStream_t st);
 
@@ -121,10 +141,10 @@ struct AttnLaunch {
   int nunits;
   const __nv_bfloat16* qkv;    // tile base
   const __nv_bfloat16* table;  // [(2M-1)^2, nh]
-  __nv_bfloat16* A;            // fwd: [T, C] out
+  __nv_bfloat16* A;            // fwd: [T, Ap] out
   float* Lt;                   // L tiles (fwd: out or nullptr; bwd: in)
   const __nv_bfloat16* dO;     // bwd: dO tiles
-  __nv_bfloat16* dqkv;         // bwd: [T, 3C] out
+  __nv_bfloat16* dqkv;         // bwd: [T, 3*Ap] out
   float* dtable;               // bwd: [(2M-1)^2, nh] float, atomics; or nullptr
   float scale;
 };

@@ -225,15 +225,18 @@ __global__ void __launch_bounds__(384, 2) attn_fwd_kernel(const __grid_constant_
     regs_times_tile<DP>(o, s, v_base, lane);
 
     const float inv0 = 1.f / sum0, inv1 = 1.f / sum1;
-    __nv_bfloat16* out0 = L.A + (long long)tok[p0] * g.C + h * g.d;
-    __nv_bfloat16* out1 = L.A + (long long)tok[p0 + 8] * g.C + h * g.d;
+    // rows of the padded attention output: DP columns per head, pad columns are exact zeros because
+    // the pad columns of v are; column d of head 0 is set to one (bias-gradient column, see fast.cuh)
+    const int Ap = g.nh * DP;
+    __nv_bfloat16* out0 = L.A + (long long)tok[p0] * Ap + h * DP;
+    __nv_bfloat16* out1 = L.A + (long long)tok[p0 + 8] * Ap + h * DP;
 #pragma unroll
     for (int jn = 0; jn < DP / 8; ++jn) {
       const int col = 8 * jn + 2 * t;
-      if (col < g.d) {
-        *reinterpret_cast<uint32_t*>(out0 + col) = pack2(o[jn][0] * inv0, o[jn][1] * inv0);
-        *reinterpret_cast<uint32_t*>(out1 + col) = pack2(o[jn][2] * inv1, o[jn][3] * inv1);
-      }
+      uint32_t w0 = pack2(o[jn][0] * inv0, o[jn][1] * inv0), w1 = pack2(o[jn][2] * inv1, o[jn][3] * inv1);
+      if (h == 0 && col == g.d) w0 = w1 = 0x00003F80u;       // (1.0, 0.0)
+      *reinterpret_cast<uint32_t*>(out0 + col) = w0;
+      *reinterpret_cast<uint32_t*>(out1 + col) = w1;
     }
     if (L.Lt != nullptr && t == 0) {
       float* lt = L.Lt + u.l_off + win * u.l_wstride + hl * 64;
@@ -273,6 +276,7 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
   }
   const int hl = warp >> 2, r0 = (warp & 3) * 16, gq = lane >> 2, t = lane & 3;
   const int h = u.h0 + hl;
+  const int Ap = g.nh * DP;                                    // row length of the padded token-major buffers
   unsigned char* Ph = Ps + (size_t)hl * 8192;
   unsigned char* dSh = dSs + (size_t)hl * 8192;
   const int p0 = r0 + gq;
@@ -352,15 +356,13 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
 #pragma unroll
       for (int j = 0; j < DP / 8; ++j) dq[j][0] = dq[j][1] = dq[j][2] = dq[j][3] = 0.f;
       regs_times_tile<DP>(dq, dp, k_base, lane);             // dQ = dS K
-      __nv_bfloat16* o0 = L.dqkv + (long long)tok[p0] * 3 * g.C + h * g.d;
-      __nv_bfloat16* o1 = L.dqkv + (long long)tok[p0 + 8] * 3 * g.C + h * g.d;
+      __nv_bfloat16* o0 = L.dqkv + (long long)tok[p0] * 3 * Ap + h * DP;
+      __nv_bfloat16* o1 = L.dqkv + (long long)tok[p0 + 8] * 3 * Ap + h * DP;
 #pragma unroll
       for (int jn = 0; jn < DP / 8; ++jn) {
         const int col = 8 * jn + 2 * t;
-        if (col < g.d) {
-          *reinterpret_cast<uint32_t*>(o0 + col) = pack2(dq[jn][0] * L.scale, dq[jn][1] * L.scale);
-          *reinterpret_cast<uint32_t*>(o1 + col) = pack2(dq[jn][2] * L.scale, dq[jn][3] * L.scale);
-        }
+        *reinterpret_cast<uint32_t*>(o0 + col) = pack2(dq[jn][0] * L.scale, dq[jn][1] * L.scale);
+        *reinterpret_cast<uint32_t*>(o1 + col) = pack2(dq[jn][2] * L.scale, dq[jn][3] * L.scale);
       }
     }
     __syncthreads();
@@ -392,17 +394,15 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
       }
     }
     {
-      __nv_bfloat16* o0 = L.dqkv + (long long)tok[p0] * 3 * g.C + g.C + h * g.d;
-      __nv_bfloat16* o1 = L.dqkv + (long long)tok[p0 + 8] * 3 * g.C + g.C + h * g.d;
+      __nv_bfloat16* o0 = L.dqkv + (long long)tok[p0] * 3 * Ap + Ap + h * DP;
+      __nv_bfloat16* o1 = L.dqkv + (long long)tok[p0 + 8] * 3 * Ap + Ap + h * DP;
 #pragma unroll
       for (int jn = 0; jn < DP / 8; ++jn) {
         const int col = 8 * jn + 2 * t;
-        if (col < g.d) {
-          *reinterpret_cast<uint32_t*>(o0 + col) = pack2(dk[jn][0], dk[jn][1]);
-          *reinterpret_cast<uint32_t*>(o1 + col) = pack2(dk[jn][2], dk[jn][3]);
-          *reinterpret_cast<uint32_t*>(o0 + g.C + col) = pack2(dv[jn][0], dv[jn][1]);
-          *reinterpret_cast<uint32_t*>(o1 + g.C + col) = pack2(dv[jn][2], dv[jn][3]);
-        }
+        *reinterpret_cast<uint32_t*>(o0 + col) = pack2(dk[jn][0], dk[jn][1]);
+        *reinterpret_cast<uint32_t*>(o1 + col) = pack2(dk[jn][2], dk[jn][3]);
+        *reinterpret_cast<uint32_t*>(o0 + Ap + col) = pack2(dv[jn][0], dv[jn][1]);
+        *reinterpret_cast<uint32_t*>(o1 + Ap + col) = pack2(dv[jn][2], dv[jn][3]);
       }
     }
     __syncthreads();   // tiles, P and dS of this window are no longer read

@@ -106,15 +106,17 @@ struct RingPos {
   }
 };
 
-// One thread of a loader set: 8-token column `lw` of every 8-row group, 16-byte chunk `pp` of the atom
-// row (copied as two 8-byte pieces: source rows are only 8-byte aligned).  Tile row r = lw + 8k has
-// (r & 7) == lw, so the swizzled destination is dst0 + 1024 k.
+// One thread of a loader set (64 threads): tile rows lw + 8k (lw = 0..7) and the 16-byte chunk `pp` of the
+// 128-byte atom row, copied as two 8-byte pieces because the caller's rows are only 8-byte aligned.
+// Consecutive lanes take consecutive chunks of the same row, so one copy instruction reads four rows
+// of 128 contiguous bytes.  Tile row r = lw + 8k has (r & 7) == lw: the swizzled destination is
+// dst0 + 1024 k.
 struct LoaderLane {
   int lw, pp;
   uint32_t dst0;
   __device__ __forceinline__ void init(int ts) {
-    lw = ts & 7;
-    pp = ts >> 3;
+    lw = ts >> 3;
+    pp = ts & 7;
     dst0 = sw128_offset(lw, pp * 8);
   }
 };
@@ -362,7 +364,7 @@ __global__ void __launch_bounds__(kThreads2, 1) gt_kernel(const __grid_constant_
   fence_proxy_async();
   if (tid == 0) {
     abort_s = 0;
-    for (int i = 0; i < 8; ++i) { mbar_init(&full[i], 2); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < 8; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], kEpi2); }
     mbar_init_fence();
   }
@@ -375,42 +377,22 @@ __global__ void __launch_bounds__(kThreads2, 1) gt_kernel(const __grid_constant_
   const long long n_tiles = (L.rows + 127) / 128;
 
   if (warp > kEpi2) {
-    // ---------------- loaders (four sets of two warps, see above)
-    const int set = (warp - kEpi2 - 1) >> 1;
-    LoaderLane ll;
-    ll.init(((warp - kEpi2 - 1) & 1) * 32 + lane);
-    const char* const srcA = reinterpret_cast<const char*>(L.A);
-    const long long row_bytes = (long long)L.lda * 2;
-    const uint32_t ringA = smem_u32(ring);
-    RingPos rp;
-    rp.init(set, S);
-    int g = set, it = 0;
-    for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
-      const long long trow = tile * 128 + ll.lw;
-      const char* const src_t = srcA + trow * row_bytes + ll.pp * 16;
-      const bool full_tile = (tile + 1) * 128 <= L.rows;
+    // ---------------- producer: one thread asks TMA for one K atom (64 columns x 128 rows, swizzled on
+    // the way in) per ring step; rows past the end of the tensor arrive as zeros
+    if (warp == kEpi2 + 1 && lane == 0) {
+      const uint32_t ringA = smem_u32(ring);
+      RingPos rp;
+      rp.init(0, S);
       bool ok = true;
-      for (; g < (it + 1) * natoms; g += kSets) {
-        const int atom = g - it * natoms;
-        if (!wait_bar_warp(&empty[rp.slot], rp.ph ^ 1, &abort_s, L.err)) { ok = false; break; }
-        const uint32_t dst = ringA + rp.slot * kAtomBytes + ll.dst0;
-        const int colb = atom * 128 + ll.pp * 16;
-        const bool v0 = colb < L.kvalid * 2, v1 = colb + 8 < L.kvalid * 2;
-        const char* src = src_t + atom * 128;
-#pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const bool rv = full_tile || trow + 8 * k < L.rows;
-          cp_async8(dst + k * 1024, rv && v0 ? src + k * 8 * row_bytes : srcA, rv && v0);
-          cp_async8(dst + k * 1024 + 8, rv && v1 ? src + k * 8 * row_bytes + 8 : srcA, rv && v1);
+      for (long long tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        for (int atom = 0; atom < natoms; ++atom) {
+          if (!wait_bar(&empty[rp.slot], rp.ph ^ 1, &abort_s, L.err)) { ok = false; break; }
+          mbar_arrive_expect_tx(&full[rp.slot], kAtomBytes);
+          tma_load_2d(ringA + rp.slot * kAtomBytes, &L.tmA, atom * 64, (int)(tile * 128), &full[rp.slot]);
+          rp.advance(1, S);
         }
-        cp_async_commit();
-        cp_async_wait(0);
-        publish(&full[rp.slot], lane);
-        rp.advance(kSets, S);
       }
-      if (!ok) break;
     }
-    cp_async_wait(0);
   } else if (warp == kEpi2) {
     if (lane == 0) {
       const uint32_t idesc = make_idesc(128, NB, 0, 0);
@@ -495,20 +477,25 @@ __global__ void __launch_bounds__(kThreads2, 1) gt_kernel(const __grid_constant_
 // ==========================================================================================
 // gr_kernel
 // ==========================================================================================
-__device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
-  asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d)
-               : "memory");
+__device__ __forceinline__ void red_add_v2(float* p, float a, float b) {
+  asm volatile("red.relaxed.gpu.global.add.v2.f32 [%0], {%1, %2};" ::"l"(p), "f"(a), "f"(b) : "memory");
+}
+// Padded index (kind, head, c) -> kind*C + head*d + c, or -1 for a pad column.
+__device__ __forceinline__ int unpad_index(int idx, int Ap, int dp, int d, int C) {
+  const int kind = idx / Ap, rem = idx - kind * Ap;
+  const int h = rem / dp, c = rem - h * dp;
+  return c < d ? kind * C + h * d + c : -1;
 }
 
 __global__ void __launch_bounds__(kThreads, 1) gr_kernel(const __grid_constant__ GRLaunch L) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = align1024(smem_raw);
   const int NP = L.NP, ratoms = NP / 64;
-  const int stage_bytes = (2 + ratoms) * 8192;
-  __shared__ uint64_t full[4], empty[4], done;
+  const int stage_bytes = (2 + ratoms) * 8192;             // [L atom 0 | L atom 1 | R atoms], 64 tokens x 64 columns each
+  __shared__ uint64_t full[8], empty[8], done;
   __shared__ uint32_t tmem_s;
   __shared__ int abort_s;
-  constexpr int S = 4;
+  const int S = L.nstages;                               // ring depth; S - 1 stages of loads stay in flight
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int mb = blockIdx.y;
@@ -518,10 +505,14 @@ __global__ void __launch_bounds__(kThreads, 1) gr_kernel(const __grid_constant__
   const long long t1 = t0 + chunk < L.rows ? t0 + chunk : L.rows;
   if (t0 >= t1) return;
   const int nst = (int)((t1 - t0 + 63) / 64);
+  // atoms TMA brings per stage, and where they go
+  const int tma_cols = L.tma_is_L ? L.M - mb * 128 : L.Ap;                 // valid columns of the TMA-fed operand here
+  const int tma_atoms = tma_cols >= (L.tma_is_L ? 128 : NP) ? (L.tma_is_L ? 2 : ratoms) : (tma_cols + 63) / 64;
+  const int tma_atoms_all = L.tma_is_L ? 2 : ratoms;
 
   if (tid == 0) {
     abort_s = 0;
-    for (int i = 0; i < S; ++i) { mbar_init(&full[i], kLoadWarps); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < S; ++i) { mbar_init(&full[i], L.use_tma ? 3 : 2); mbar_init(&empty[i], 1); }   // two warps of a set (+ the TMA request)
     mbar_init(&done, 1);
     mbar_init_fence();
   }
@@ -533,116 +524,123 @@ __global__ void __launch_bounds__(kThreads, 1) gr_kernel(const __grid_constant__
   const uint32_t tmem = tmem_s;
 
   if (warp > kEpiWarps) {
-    const int lw = warp - kEpiWarps - 1;
-    const int lcol = mb * 128 + lane * 4;
-    constexpr int lag = 2;
-    // Stage row r = lw + 8k has (r & 7) == lw: every piece's swizzled destination is a per-lane
-    // constant plus 1024 bytes per k.  Pieces that never change (K/M padding, the ones column that
-    // turns the GEMM into a column sum of L) are written once per stage buffer, before the loop.
-    const uint32_t dL = (uint32_t)((lane >> 4) * 8192) + sw128_offset(lw, (lane & 15) * 4);
-    const bool lvalid = lcol < L.mvalid;
-    uint32_t dR[2];
-    int rkind[2];                                 // 0 = data, 1 = ones column, 2 = zero padding, 3 = outside the stage
-#pragma unroll
-    for (int pi = 0; pi < 2; ++pi) {
-      const int col = (lane + 32 * pi) * 4;
-      dR[pi] = (uint32_t)(2 * 8192 + (col >> 6) * 8192) + sw128_offset(lw, col & 63);
-      rkind[pi] = col >= NP ? 3 : (col < L.nvalid ? 0 : (col == L.nvalid ? 1 : 2));
-    }
-    for (int sgi = 0; sgi < S; ++sgi) {
+    // ---------------- loaders: four sets of two warps; set q fills ring steps q, q+4, ...  Its leader
+    // asks TMA for the padded operand's 64-token boxes, all 64 threads copy the caller's rows in
+    // 8-byte pieces, and the step is published as soon as the set's own copies have landed.
+    const int set = (warp - kEpiWarps - 1) >> 1;
+    const int ts = ((warp - kEpiWarps - 1) & 1) * 32 + lane;
+    LoaderLane ll;
+    ll.init(ts);
+    const int copy_base = L.tma_is_L ? 2 * 8192 : 0;                       // copy-fed operand inside a stage
+    const int copy_atoms = L.tma_is_L ? ratoms : 2;
+    const int copy_col0 = L.tma_is_L ? 0 : mb * 128;                       // first column of the copy-fed operand here
+    // Pieces that never change (padding, the ones column, atoms TMA never touches) are written once per
+    // stage buffer, before the loop.
+    for (int sgi = set; sgi < S; sgi += kSets) {
       unsigned char* base = sm + (size_t)sgi * stage_bytes;
+      for (int a = 0; a < copy_atoms; ++a)
+        for (int half = 0; half < 2; ++half) {
+          const int col = copy_col0 + a * 64 + ll.pp * 8 + half * 4;
+          if (col < L.pvalid) continue;
+          const uint2 val = make_uint2((L.tma_is_L && col == L.pvalid) ? 0x3F80u : 0u, 0u);
 #pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        if (!lvalid) *reinterpret_cast<uint2*>(base + dL + k * 1024) = make_uint2(0u, 0u);
-#pragma unroll
-        for (int pi = 0; pi < 2; ++pi)
-          if (rkind[pi] == 1 || rkind[pi] == 2)
-            *reinterpret_cast<uint2*>(base + dR[pi] + k * 1024) = make_uint2(rkind[pi] == 1 ? 0x3F80u : 0u, 0u);
+          for (int k = 0; k < 8; ++k)
+            *reinterpret_cast<uint2*>(base + copy_base + a * 8192 + ll.dst0 + k * 1024 + half * 8) = val;
+        }
+      for (int a = tma_atoms; a < tma_atoms_all; ++a) {
+        unsigned char* at = base + (L.tma_is_L ? 0 : 2 * 8192) + a * 8192;
+        for (int e = ts; e < 8192 / 16; e += 64) reinterpret_cast<uint4*>(at)[e] = make_uint4(0u, 0u, 0u, 0u);
       }
     }
-    const char* const srcL = reinterpret_cast<const char*>(L.L);
-    const char* const srcR = reinterpret_cast<const char*>(L.R);
-    const long long lrow = (long long)L.ldl * 2, rrow = (long long)L.ldr * 2;
-    int st = 0, ph = 0, n = 0, pub = 0;
-    bool ok = true;
-    for (int s = 0; s < nst; ++s) {
-      if (!wait_bar_warp(&empty[st], ph ^ 1, &abort_s, L.err)) { ok = false; break; }
-      const uint32_t sS = smem_u32(sm + (size_t)st * stage_bytes);
-      const long long tb = t0 + (long long)s * 64 + lw;
-      const char* pl = srcL + tb * lrow + lcol * 2;
-      const char* pr = srcR + tb * rrow + lane * 8;
-      if (tb - lw + 64 <= t1) {
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          if (lvalid) cp_async8(sS + dL + k * 1024, pl + k * 8 * lrow, true);
-          if (rkind[0] == 0) cp_async8(sS + dR[0] + k * 1024, pr + k * 8 * rrow, true);
-          if (rkind[1] == 0) cp_async8(sS + dR[1] + k * 1024, pr + k * 8 * rrow + 256, true);
+    const char* const srcP = reinterpret_cast<const char*>(L.P);
+    const long long prow = (long long)L.ldp * 2;
+    RingPos rp;
+    rp.init(set, S);
+    for (int s = set; s < nst; s += kSets) {
+      if (!wait_bar_warp(&empty[rp.slot], rp.ph ^ 1, &abort_s, L.err)) break;
+      const uint32_t sS = smem_u32(sm + (size_t)rp.slot * stage_bytes);
+      const long long tb = t0 + (long long)s * 64;
+      if (L.use_tma) {
+        if (ts == 0) {
+          // the TMA-fed operand; rows past the end of the tensor arrive as zeros
+          mbar_arrive_expect_tx(&full[rp.slot], (uint32_t)tma_atoms * 8192u);
+          for (int a = 0; a < tma_atoms; ++a)
+            tma_load_2d(sS + (L.tma_is_L ? 0 : 2 * 8192) + a * 8192, &L.tm, (L.tma_is_L ? mb * 128 : 0) + a * 64, (int)tb,
+                        &full[rp.slot]);
         }
       } else {
+        // the padded operand by 16-byte copies (its rows are 16-byte aligned)
+        const int qc0 = (L.tma_is_L ? mb * 128 : 0) + ll.pp * 8;
+        const char* q = reinterpret_cast<const char*>(L.Q) + ((tb + ll.lw) * (long long)L.qcols + qc0) * 2;
+        const uint32_t qd = sS + (L.tma_is_L ? 0 : 2 * 8192) + ll.dst0;
+        for (int a = 0; a < tma_atoms; ++a) {
+          const bool cv = qc0 + a * 64 < L.qcols;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const bool v = cv && tb + ll.lw + 8 * k < L.rows;
+            cp_async16(qd + a * 8192 + k * 1024, v ? q + ((long long)k * 8 * L.qcols + a * 64) * 2 : (const char*)L.Q, v);
+          }
+        }
+      }
+      const char* pp = srcP + (tb + ll.lw) * prow + (copy_col0 + ll.pp * 8) * 2;
+      const bool whole = tb + 64 <= t1;
+      for (int a = 0; a < copy_atoms; ++a) {
+        const int col = copy_col0 + a * 64 + ll.pp * 8;
+        const bool v0 = col < L.pvalid, v1 = col + 4 < L.pvalid;
+        if (!v0) break;
+        const uint32_t dst = sS + copy_base + a * 8192 + ll.dst0;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-          const bool tv = tb + 8 * k < t1;
-          if (lvalid) cp_async8(sS + dL + k * 1024, tv ? pl + k * 8 * lrow : srcL, tv);
-          if (rkind[0] == 0) cp_async8(sS + dR[0] + k * 1024, tv ? pr + k * 8 * rrow : srcR, tv);
-          if (rkind[1] == 0) cp_async8(sS + dR[1] + k * 1024, tv ? pr + k * 8 * rrow + 256 : srcR, tv);
+          const bool tv = whole || tb + ll.lw + 8 * k < t1;
+          const char* src = pp + k * 8 * prow + a * 128;
+          cp_async8(dst + k * 1024, tv ? src : srcP, tv);
+          if (v1) cp_async8(dst + k * 1024 + 8, tv ? src + 8 : srcP, tv);
         }
       }
       cp_async_commit();
-      if (++st == S) { st = 0; ph ^= 1; }
-      if (++n > lag) {
-        cp_async_wait(lag);
-        publish(&full[pub], lane);
-        if (++pub == S) pub = 0;
-      }
+      cp_async_wait(0);
+      publish(&full[rp.slot], lane);
+      rp.advance(kSets, S);
     }
-    {
-      int left = n < lag ? n : lag;
-      while (left > 0) {
-        cp_async_wait(left - 1);
-        if (ok) publish(&full[pub], lane);
-        if (++pub == S) pub = 0;
-        --left;
-      }
-    }
+    cp_async_wait(0);
   } else if (warp == kEpiWarps) {
     if (lane == 0) {
       const uint32_t idesc = make_idesc(128, NP, 1, 1);
-      int st = 0, ph = 0;
+      RingPos rp;
+      rp.init(0, S);
       bool ok = true;
       for (int s = 0; s < nst; ++s) {
-        if (!wait_bar(&full[st], ph, &abort_s, L.err)) { ok = false; break; }
+        if (!wait_bar(&full[rp.slot], rp.ph, &abort_s, L.err)) { ok = false; break; }
         fence_after_sync();
-        const uint32_t lAddr = smem_u32(sm + (size_t)st * stage_bytes), rAddr = lAddr + 2 * 8192;
+        const uint32_t lAddr = smem_u32(sm + (size_t)rp.slot * stage_bytes), rAddr = lAddr + 2 * 8192;
+        const uint64_t ad = make_desc(lAddr, 8192, 1024), bd = make_desc(rAddr, 8192, 1024);
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          const uint64_t ad = make_desc(lAddr + kk * 2048, 8192, 1024);
-          const uint64_t bd = make_desc(rAddr + kk * 2048, 8192, 1024);
-          mma_bf16(tmem, ad, bd, idesc, (s | kk) != 0);
-        }
-        commit(&empty[st]);
-        if (++st == S) { st = 0; ph ^= 1; }
+        for (int kk = 0; kk < 4; ++kk) mma_bf16(tmem, ad + kk * 128, bd + kk * 128, idesc, (s | kk) != 0);
+        commit(&empty[rp.slot]);
+        rp.advance(1, S);
       }
       if (ok) commit(&done);
     }
   } else {
     if (wait_bar_warp(&done, 0, &abort_s, L.err)) {
       fence_after_sync();
-      const int m = mb * 128 + tid;
+      const int mi = mb * 128 + tid;                                  // index in the M space
+      const int m = L.tma_is_L ? (mi < L.M ? unpad_index(mi, L.Ap, L.dp, L.d, L.C) : -1) : (mi < L.M ? mi : -1);
+      const int ones = L.tma_is_L ? L.pvalid : (L.d < L.dp ? L.d : -1);   // N index of the ones column
       for (int c0 = 0; c0 < NP; c0 += 32) {
-        if (c0 > L.nvalid) break;
         uint32_t v[32];
         tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + c0, v);
         tmem_ld_wait();
-        if (m < L.mvalid) {
-          float* orow = L.out + (long long)m * L.nvalid;
+        if (m >= 0) {
+          float* orow = L.out + (long long)m * L.C;
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            const int n = c0 + j;
-            if (n + 3 < L.nvalid) {
-              red_add_v4(orow + n, __uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
-                         __uint_as_float(v[j + 3]));
-            } else if (n == L.nvalid && L.colsum != nullptr) {
-              atomicAdd(L.colsum + m, __uint_as_float(v[j]));
+          for (int j = 0; j < 32; j += 2) {
+            const int ni = c0 + j;
+            if (ni == ones) {
+              if (L.colsum != nullptr) atomicAdd(L.colsum + m, __uint_as_float(v[j]));
+            } else {
+              const int n = L.tma_is_L ? (ni + 1 < L.C ? ni : -1) : (ni < L.Ap ? unpad_index(ni, L.Ap, L.dp, L.d, L.C) : -1);
+              if (n >= 0) red_add_v2(orow + n, __uint_as_float(v[j]), __uint_as_float(v[j + 1]));
             }
           }
         }
@@ -677,10 +675,13 @@ __global__ void prep_kernel(const __grid_constant__ PrepJobs J) {
     } else if (p.mode == PREP_PROJ_T) {  // row n = (head, c) -> input channel of W_proj; k = output channel
       const int h = p.h0 + n / p.dp, c = n % p.dp;
       if (c < p.d && k < C) val = __bfloat162float(p.W[(long long)k * C + h * p.d + c]);
-    } else if (p.mode == PREP_PROJ) {    // row n = output channel n0+n of W_proj; k = input channel
-      if (p.n0 + n < C && k < C) val = __bfloat162float(p.W[(long long)(p.n0 + n) * C + k]);
-    } else {                             // PREP_QKV_T: row n = input channel n0+n; k = row of W_qkv
-      if (p.n0 + n < C && k < 3 * C) val = __bfloat162float(p.W[(long long)k * C + p.n0 + n]);
+    } else if (p.mode == PREP_PROJ) {    // row n = output channel n0+n of W_proj; k = padded (head, c) input index
+      const int h = k / p.dp, c = k % p.dp;
+      if (p.n0 + n < C && k < p.Ap && c < p.d) val = __bfloat162float(p.W[(long long)(p.n0 + n) * C + h * p.d + c]);
+    } else {                             // PREP_QKV_T: row n = input channel n0+n; k = padded (kind, head, c) row of W_qkv
+      const int kind = k / p.Ap, rem = k % p.Ap, h = rem / p.dp, c = rem % p.dp;
+      if (p.n0 + n < C && kind < 3 && c < p.d)
+        val = __bfloat162float(p.W[(long long)(kind * C + h * p.d + c) * C + p.n0 + n]);
     }
     *reinterpret_cast<__nv_bfloat16*>(p.img + (size_t)(k >> 6) * p.NT * 128 + sw128_offset(n, k & 63)) =
         __float2bfloat16_rn(val);
@@ -758,6 +759,29 @@ size_t gt_smem_bytes(int natoms, int NB, int nstages) {
   return 1024 + (size_t)natoms * NB * 128 + (size_t)nstages * kAtomBytes + (size_t)128 * NB * 2 + (size_t)NB * 4 + 64;
 }
 
+int make_tmap(CUtensorMap* tm, const void* base, long long rows, int cols, int box_rows) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess || p == nullptr)
+      return check_launch() ? GSWA_ERR_CUDA : GSWA_ERR_CUDA;
+    fn = reinterpret_cast<EncodeFn>(p);
+  }
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+  const cuuint32_t es[2] = {1u, 1u};
+  const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? GSWA_OK : GSWA_ERR_CUDA;
+}
+
 int launch_gt(const GTLaunch& L, int nsplits, cudaStream_t st, const char* name) {
   const size_t smem = gt_smem_bytes(L.natoms, L.NB, L.nstages);
   if (cudaFuncSetAttribute(gt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
@@ -771,11 +795,15 @@ int launch_gt(const GTLaunch& L, int nsplits, cudaStream_t st, const char* name)
 }
 
 int launch_gr(const GRLaunch& L, cudaStream_t st, const char* name) {
-  const size_t smem = 1024 + (size_t)4 * (2 + L.NP / 64) * 8192 + 64;
+  GRLaunch Lc = L;
+  Lc.nstages = (int)((215 * 1024) / ((size_t)(2 + L.NP / 64) * 8192));
+  if (Lc.nstages > 6) Lc.nstages = 6;
+  if (Lc.nstages < 3) return GSWA_ERR_UNSUPPORTED;
+  const size_t smem = 1024 + (size_t)Lc.nstages * (2 + L.NP / 64) * 8192 + 64;
   if (cudaFuncSetAttribute(gr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return check_launch();
-  const int mblocks = (L.mvalid + 127) / 128;
-  { KernelScope ks_(name, st); gr_kernel<<<dim3(L.nsplit, mblocks), kThreads, smem, st>>>(L); }
+  const int mblocks = (L.M + 127) / 128;
+  { KernelScope ks_(name, st); gr_kernel<<<dim3(L.nsplit, mblocks), kThreads, smem, st>>>(Lc); }
   return check_launch();
 }
 

@@ -406,6 +406,10 @@ int generic_backward(const Plan& p, const void* x, const void* w_qkv, const void
                         (const bf*)dy, (bf*)dx, dw_qkv, db_qkv, dw_proj, db_proj, dtable, (char*)scratch, st);
 }
 
+int launch_colsum_bf16(const __nv_bfloat16* G, long long rows, int cols, long long ld, float* out, cudaStream_t st) {
+  return launch_colsum<__nv_bfloat16>(G, rows, cols, ld, out, st);
+}
+
 int launch_index_maps(const Plan& p, int group, int32_t* win, int32_t* slot, int32_t* region, int32_t* token_of,
                       int32_t* rel, cudaStream_t st) {
   const int n = max(p.H * p.W, p.N * p.N);

@@ -25,7 +25,8 @@ struct Plan {
   int fast;                    // 1 = bf16 tensor-core path, 0 = generic CUDA-core path
   // fast-path geometry
   int dp;                      // head dim padded to an MMA-friendly width (16 or 32)
-  int Cp;                      // C padded to a multiple of 64 (GEMM K / row pitch of padded activations)
+  int Cp;                      // C padded to a multiple of 64 (K of the GEMMs that read the caller's rows)
+  int Ap;                      // heads * dp: row length of the padded attention output
   // byte offsets inside `saved`
   size_t off_qkv, off_A, off_L, saved_bytes;
   size_t fwd_scratch, infer_scratch, bwd_scratch;
@@ -54,6 +55,7 @@ int generic_forward(const Plan& p, const void* x, const void* w_qkv, const void*
 int generic_backward(const Plan& p, const void* x, const void* w_qkv, const void* w_proj, const void* table,
                      const void* saved, const void* dy, void* dx, float* dw_qkv, float* db_qkv, float* dw_proj,
                      float* db_proj, float* dtable, void* scratch, cudaStream_t st);
+int launch_colsum_bf16(const __nv_bfloat16* G, long long rows, int cols, long long ld, float* out, cudaStream_t st);
 int launch_index_maps(const Plan& p, int group, int32_t* win, int32_t* slot, int32_t* region, int32_t* token_of,
                       int32_t* rel, cudaStream_t st);
 

@@ -105,16 +105,25 @@ __device__ __forceinline__ void cp_async8(uint32_t dst_smem, const void* src, bo
   const uint32_t n = valid ? 8u : 0u;
   asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst_smem), "l"(src), "r"(n) : "memory");
 }
+__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src, bool valid) {
+  const uint32_t n = valid ? 16u : 0u;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(n) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-// Waits until at most `n` of this thread's committed groups are still in flight (n <= 3).
+// Waits until at most `n` of this thread's committed groups are still in flight (n <= 4).
 __device__ __forceinline__ void cp_async_wait(int n) {
   switch (n) {
     case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
     case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
     case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
-    default: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+    case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+    default: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
   }
 }
+
+// ---- TMA: one 2-D tile of a tensor map into shared memory; completion is counted in bytes on `bar`
+// (the issuing thread first arrives with mbar_arrive_expect_tx).  No multicast.
+__device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const void* tmap, int x, int y, uint64_t* bar);
 
 // ---- mbarriers (shared::cta), every wait bounded
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -143,6 +152,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32
     if (i > 64) __nanosleep(32);
   }
   return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const void* tmap, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(smem_dst),
+      "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
 }
 
 }  // namespace umma
