@@ -217,7 +217,7 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
     w.out = qkv + geo.qkv_off[u.g] + (long long)(u.h0 - p.gh0[u.g]) * 3 * 64 * p.dp;
     w.win_stride = (long long)p.gh[u.g] * 3 * 64 * p.dp;
     w.nchunks = u.nheads; w.cw = 3 * p.dp; w.q_every3 = 1;
-    w.qscale = 1.0f / sqrtf((float)p.d);
+    w.qscale = 1.4426950408889634f / sqrtf((float)p.d);   // d^-1/2 and log2(e): the attention kernels work in the log2 domain
   }
   if ((rc = launch_gw(gw, nu, p.Cp, p.dp, st, "qkv_gemm"))) return rc;
 

@@ -45,6 +45,19 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
 
 constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
 
+__device__ __forceinline__ float ex2(float x) {          // 2^x, one MUFU instruction; 2^-inf = 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void stsm_x4(uint32_t addr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3) {
+  asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
+               : "memory");
+}
+__device__ __forceinline__ void stsm_x2(uint32_t addr, uint32_t r0, uint32_t r1) {
+  asm volatile("stmatrix.sync.aligned.m8n8.x2.shared.b16 [%0], {%1,%2};" ::"r"(addr), "r"(r0), "r"(r1) : "memory");
+}
+
 // [64][64] bf16 matrices (P, dS): 128-byte rows, chunk ^= row & 7.
 __device__ __forceinline__ uint32_t sq_off(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
 
@@ -97,6 +110,50 @@ __device__ __forceinline__ void regs_times_tile(float (*acc)[4], const float (*p
   }
 }
 
+__device__ __forceinline__ void set_word(uint4& v, int i, uint32_t w) {
+  if (i == 0) v.x = w; else if (i == 1) v.y = w; else if (i == 2) v.z = w; else v.w = w;
+}
+
+// Writes a warp's 16 x DP accumulator tile (rows gq, gq+8 of the mma fragment) to rows of a padded
+// token-major buffer: the tile is first laid out in the warp's 16 x DP staging block (stmatrix), then
+// every lane moves 16 bytes per row so that one store instruction covers whole 2*DP-byte row pieces.
+// `row0` / `row1` are the global addresses of the lane's two rows (fragment rows gq and gq + 8).
+template <int DP>
+__device__ __forceinline__ void store_tile(unsigned char* stg, const float (*acc)[4], float scale, unsigned char* row0,
+                                           unsigned char* row1, int lane, int ones_col) {
+  const uint32_t sa = smem_u32(stg);
+  const int m = lane >> 3;
+#pragma unroll
+  for (int jn = 0; jn < DP / 8; jn += 2) {
+    const int row = (m & 1) * 8 + (lane & 7), chunk = jn + (m >> 1);
+    stsm_x4(sa + tile_off<DP>(row, chunk), pack2(acc[jn][0] * scale, acc[jn][1] * scale),
+            pack2(acc[jn][2] * scale, acc[jn][3] * scale), pack2(acc[jn + 1][0] * scale, acc[jn + 1][1] * scale),
+            pack2(acc[jn + 1][2] * scale, acc[jn + 1][3] * scale));
+  }
+  __syncwarp();
+  if constexpr (DP == 32) {
+    const int gq = lane >> 2, t = lane & 3;
+    uint4 v0 = *reinterpret_cast<const uint4*>(stg + tile_off<DP>(gq, t));
+    uint4 v1 = *reinterpret_cast<const uint4*>(stg + tile_off<DP>(gq + 8, t));
+    if (ones_col >= 0 && (ones_col >> 3) == t) {
+      set_word(v0, (ones_col & 7) >> 1, 0x00003F80u);        // (1.0, 0.0)
+      set_word(v1, (ones_col & 7) >> 1, 0x00003F80u);
+    }
+    *reinterpret_cast<uint4*>(row0 + t * 16) = v0;
+    *reinterpret_cast<uint4*>(row1 + t * 16) = v1;
+  } else {
+    // DP == 16: 16 rows x 2 chunks, one chunk per lane; the lane's row pointer comes from a neighbour
+    const int r = lane >> 1, c = lane & 1;
+    uint4 v = *reinterpret_cast<const uint4*>(stg + tile_off<DP>(r, c));
+    if (ones_col >= 0 && (ones_col >> 3) == c) set_word(v, (ones_col & 7) >> 1, 0x00003F80u);
+    // row pointers live in lanes with gq == r (rows 0..7: row0 of lane 4r) or gq == r - 8 (row1 of lane 4(r-8))
+    const unsigned long long a0 = __shfl_sync(0xffffffffu, (unsigned long long)row0, (r & 7) * 4);
+    const unsigned long long a1 = __shfl_sync(0xffffffffu, (unsigned long long)row1, (r & 7) * 4);
+    *reinterpret_cast<uint4*>((r < 8 ? a0 : a1) + c * 16) = v;
+  }
+  __syncwarp();
+}
+
 struct WinCtx {
   int b, wi, wj;
   bool masked;
@@ -119,7 +176,7 @@ __device__ __forceinline__ WinCtx window_setup(const FastGeom& g, int s, long lo
   return c;
 }
 
-// Adds the relative-position bias, applies the mask and moves the scores to the log2 domain.
+// Adds the relative-position bias and applies the mask (scores are in the log2 domain throughout).
 __device__ __forceinline__ void bias_and_mask(float (*s)[4], const float* tab, const unsigned char* reg, bool masked,
                                               int p0, int t) {
   const int pa0 = p0 >> 3, pc0 = p0 & 7;   // rows p0 and p0 + 8: same column in the window, next row
@@ -129,7 +186,7 @@ __device__ __forceinline__ void bias_and_mask(float (*s)[4], const float* tab, c
     for (int e = 0; e < 4; ++e) {
       const int pa = pa0 + (e >> 1), qc = 2 * t + (e & 1);
       const int rel = (pa - j + 7) * 15 + (pc0 - qc + 7);
-      s[j][e] = (s[j][e] + tab[rel]) * kLog2e;
+      s[j][e] += tab[rel];                  // q and the table are already scaled by log2(e)
     }
   }
   if (masked) {
@@ -164,11 +221,13 @@ __global__ void __launch_bounds__(384, 2) attn_fwd_kernel(const __grid_constant_
   int* tok2 = reinterpret_cast<int*>(tab + nh_u * 225);
   unsigned char* reg2 = reinterpret_cast<unsigned char*>(tok2 + 128);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  unsigned char* ostg = sm + 2 * (size_t)tile_bytes + (((size_t)nh_u * 225 * 4 + 128 * 4 + 128 + 15) & ~(size_t)15) +
+                        (size_t)warp * 16 * DP * 2;                 // this warp's 16 x DP output staging block
   const int nt = nh_u * 128;
   if (tid >= nt) return;
 
   for (int e = tid; e < nh_u * 225; e += nt)
-    tab[e] = __bfloat162float(L.table[(e % 225) * g.nh + u.h0 + e / 225]);
+    tab[e] = __bfloat162float(L.table[(e % 225) * g.nh + u.h0 + e / 225]) * kLog2e;
   const int hl = warp >> 2, r0 = (warp & 3) * 16, gq = lane >> 2, t = lane & 3;
   const int p0 = r0 + gq;
   const int h = u.h0 + hl;
@@ -207,10 +266,10 @@ __global__ void __launch_bounds__(384, 2) attn_fwd_kernel(const __grid_constant_
     float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      s[j][0] = exp2f(s[j][0] - m0);
-      s[j][1] = exp2f(s[j][1] - m0);
-      s[j][2] = exp2f(s[j][2] - m1);
-      s[j][3] = exp2f(s[j][3] - m1);
+      s[j][0] = ex2(s[j][0] - m0);
+      s[j][1] = ex2(s[j][1] - m0);
+      s[j][2] = ex2(s[j][2] - m1);
+      s[j][3] = ex2(s[j][3] - m1);
       sum0 += s[j][0] + s[j][1];
       sum1 += s[j][2] + s[j][3];
     }
@@ -224,20 +283,17 @@ __global__ void __launch_bounds__(384, 2) attn_fwd_kernel(const __grid_constant_
     for (int j = 0; j < DP / 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
     regs_times_tile<DP>(o, s, v_base, lane);
 
-    const float inv0 = 1.f / sum0, inv1 = 1.f / sum1;
     // rows of the padded attention output: DP columns per head, pad columns are exact zeros because
     // the pad columns of v are; column d of head 0 is set to one (bias-gradient column, see fast.cuh)
-    const int Ap = g.nh * DP;
-    __nv_bfloat16* out0 = L.A + (long long)tok[p0] * Ap + h * DP;
-    __nv_bfloat16* out1 = L.A + (long long)tok[p0 + 8] * Ap + h * DP;
+    const float inv0 = 1.f / sum0, inv1 = 1.f / sum1;
 #pragma unroll
     for (int jn = 0; jn < DP / 8; ++jn) {
-      const int col = 8 * jn + 2 * t;
-      uint32_t w0 = pack2(o[jn][0] * inv0, o[jn][1] * inv0), w1 = pack2(o[jn][2] * inv1, o[jn][3] * inv1);
-      if (h == 0 && col == g.d) w0 = w1 = 0x00003F80u;       // (1.0, 0.0)
-      *reinterpret_cast<uint32_t*>(out0 + col) = w0;
-      *reinterpret_cast<uint32_t*>(out1 + col) = w1;
+      o[jn][0] *= inv0; o[jn][1] *= inv0; o[jn][2] *= inv1; o[jn][3] *= inv1;
     }
+    const int Ap = g.nh * DP;
+    store_tile<DP>(ostg, o, 1.f, reinterpret_cast<unsigned char*>(L.A + (long long)tok[p0] * Ap + h * DP),
+                   reinterpret_cast<unsigned char*>(L.A + (long long)tok[p0 + 8] * Ap + h * DP), lane,
+                   (h == 0 && g.d < DP) ? g.d : -1);
     if (L.Lt != nullptr && t == 0) {
       float* lt = L.Lt + u.l_off + win * u.l_wstride + hl * 64;
       lt[p0] = m0 * kLn2 + logf(sum0);
@@ -267,11 +323,13 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
   int* tok2 = reinterpret_cast<int*>(hist + nh_u * 225);       // [2][64]
   unsigned char* reg2 = reinterpret_cast<unsigned char*>(tok2 + 128);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  unsigned char* ostg = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(reg2 + 128) + 15) & ~(uintptr_t)15) +
+                        (size_t)warp * 16 * DP * 2;              // this warp's 16 x DP output staging block
   const int nt = nh_u * 128;
   if (tid >= nt) return;
 
   for (int e = tid; e < nh_u * 225; e += nt) {
-    tab[e] = __bfloat162float(L.table[(e % 225) * g.nh + u.h0 + e / 225]);
+    tab[e] = __bfloat162float(L.table[(e % 225) * g.nh + u.h0 + e / 225]) * kLog2e;
     hist[e] = 0.f;
   }
   const int hl = warp >> 2, r0 = (warp & 3) * 16, gq = lane >> 2, t = lane & 3;
@@ -319,10 +377,10 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
     const float l0 = Lrow[hl * 64 + p0] * kLog2e, l1 = Lrow[hl * 64 + p0 + 8] * kLog2e;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      s[j][0] = exp2f(s[j][0] - l0);
-      s[j][1] = exp2f(s[j][1] - l0);
-      s[j][2] = exp2f(s[j][2] - l1);
-      s[j][3] = exp2f(s[j][3] - l1);
+      s[j][0] = ex2(s[j][0] - l0);
+      s[j][1] = ex2(s[j][1] - l0);
+      s[j][2] = ex2(s[j][2] - l1);
+      s[j][3] = ex2(s[j][3] - l1);
     }
     float dp[8][4];
     qk_scores<DP>(dp, do_base, v_base, r0, lane);          // dP = dO V^T
@@ -346,24 +404,28 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
       dsum[j][1] += dp[j][1];
       dsum[j][2] += dp[j][2];
       dsum[j][3] += dp[j][3];
-      *reinterpret_cast<uint32_t*>(Ph + sq_off(p0, j) + t * 4) = pack2(s[j][0], s[j][1]);
-      *reinterpret_cast<uint32_t*>(Ph + sq_off(p0 + 8, j) + t * 4) = pack2(s[j][2], s[j][3]);
-      *reinterpret_cast<uint32_t*>(dSh + sq_off(p0, j) + t * 4) = pack2(dp[j][0], dp[j][1]);
-      *reinterpret_cast<uint32_t*>(dSh + sq_off(p0 + 8, j) + t * 4) = pack2(dp[j][2], dp[j][3]);
     }
+    {
+      // P and dS cross to the key-major phase through shared memory: four 8x8 blocks per stmatrix
+      const int m = lane >> 3, srow = r0 + (m & 1) * 8 + (lane & 7);
+      const uint32_t pa = smem_u32(Ph), da = smem_u32(dSh);
+#pragma unroll
+      for (int j = 0; j < 8; j += 2) {
+        const uint32_t off = sq_off(srow, j + (m >> 1));
+        stsm_x4(pa + off, pack2(s[j][0], s[j][1]), pack2(s[j][2], s[j][3]), pack2(s[j + 1][0], s[j + 1][1]),
+                pack2(s[j + 1][2], s[j + 1][3]));
+        stsm_x4(da + off, pack2(dp[j][0], dp[j][1]), pack2(dp[j][2], dp[j][3]), pack2(dp[j + 1][0], dp[j + 1][1]),
+                pack2(dp[j + 1][2], dp[j + 1][3]));
+      }
+    }
+    unsigned char* const drow0 = reinterpret_cast<unsigned char*>(L.dqkv + (long long)tok[p0] * 3 * Ap + h * DP);
+    unsigned char* const drow1 = reinterpret_cast<unsigned char*>(L.dqkv + (long long)tok[p0 + 8] * 3 * Ap + h * DP);
     {
       float dq[DP / 8][4];
 #pragma unroll
       for (int j = 0; j < DP / 8; ++j) dq[j][0] = dq[j][1] = dq[j][2] = dq[j][3] = 0.f;
       regs_times_tile<DP>(dq, dp, k_base, lane);             // dQ = dS K
-      __nv_bfloat16* o0 = L.dqkv + (long long)tok[p0] * 3 * Ap + h * DP;
-      __nv_bfloat16* o1 = L.dqkv + (long long)tok[p0 + 8] * 3 * Ap + h * DP;
-#pragma unroll
-      for (int jn = 0; jn < DP / 8; ++jn) {
-        const int col = 8 * jn + 2 * t;
-        *reinterpret_cast<uint32_t*>(o0 + col) = pack2(dq[jn][0] * L.scale, dq[jn][1] * L.scale);
-        *reinterpret_cast<uint32_t*>(o1 + col) = pack2(dq[jn][2] * L.scale, dq[jn][3] * L.scale);
-      }
+      store_tile<DP>(ostg, dq, L.scale, drow0, drow1, lane, -1);
     }
     __syncthreads();
 
@@ -393,18 +455,9 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
         mma16816(dk[2 * jn + 1], ad, b[2], b[3]);
       }
     }
-    {
-      __nv_bfloat16* o0 = L.dqkv + (long long)tok[p0] * 3 * Ap + Ap + h * DP;
-      __nv_bfloat16* o1 = L.dqkv + (long long)tok[p0 + 8] * 3 * Ap + Ap + h * DP;
-#pragma unroll
-      for (int jn = 0; jn < DP / 8; ++jn) {
-        const int col = 8 * jn + 2 * t;
-        *reinterpret_cast<uint32_t*>(o0 + col) = pack2(dk[jn][0], dk[jn][1]);
-        *reinterpret_cast<uint32_t*>(o1 + col) = pack2(dk[jn][2], dk[jn][3]);
-        *reinterpret_cast<uint32_t*>(o0 + Ap + col) = pack2(dv[jn][0], dv[jn][1]);
-        *reinterpret_cast<uint32_t*>(o1 + Ap + col) = pack2(dv[jn][2], dv[jn][3]);
-      }
-    }
+    // q was stored scaled by log2(e) (the scores live in the log2 domain): dK = dS^T q takes it back out
+    store_tile<DP>(ostg, dk, kLn2, drow0 + Ap * 2, drow1 + Ap * 2, lane, -1);
+    store_tile<DP>(ostg, dv, 1.f, drow0 + Ap * 4, drow1 + Ap * 4, lane, -1);
     __syncthreads();   // tiles, P and dS of this window are no longer read
   }
   cp_async_wait_all();
@@ -425,10 +478,13 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
 }
 
 template <int DP>
-size_t fwd_smem(int nheads) { return (size_t)2 * nheads * 3 * 64 * DP * 2 + (size_t)nheads * 225 * 4 + 128 * 4 + 128 + 128; }
+size_t fwd_smem(int nheads) {
+  return (size_t)2 * nheads * 3 * 64 * DP * 2 + (size_t)nheads * 225 * 4 + 128 * 4 + 128 + 128 + (size_t)nheads * 4 * 16 * DP * 2;
+}
 template <int DP>
 size_t bwd_smem(int nheads) {
-  return (size_t)2 * nheads * 4 * 64 * DP * 2 + (size_t)nheads * 2 * 8192 + (size_t)nheads * (2 * 225 + 2 * 64) * 4 + 128 * 4 + 128 + 128;
+  return (size_t)2 * nheads * 4 * 64 * DP * 2 + (size_t)nheads * 2 * 8192 + (size_t)nheads * (2 * 225 + 2 * 64) * 4 + 128 * 4 + 128 + 128 +
+         (size_t)nheads * 4 * 16 * DP * 2;
 }
 
 template <int DP>
