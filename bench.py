@@ -106,6 +106,20 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def max_over_ranks(value: float) -> float:
+    """Largest `value` over all ranks of the default process group (the value itself without one).  Batch items
+    are independent, so ranks exchange nothing on the data path; this reduction of the timings is the only
+    collective of a multi-GPU run."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([float(value)], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def workload_config(cfg: LayerConfig):
     return {"workload": "%s: x[%d,%d,%d,%d] %s, %d heads (dim %d), groups %s shifts %s, window %d, %s" % (
         cfg.name, cfg.B, cfg.H, cfg.W, cfg.C, cfg.dtype, cfg.num_heads, cfg.head_dim, list(cfg.group_heads),
@@ -286,10 +300,7 @@ def run_ours(args, cfg):
     launches = gb.gswa_launch_count() - n0
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop(t0, t1) if sampler else None
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms)
     ms_step = ms / args.steps
     value = world * cfg.tokens / (ms_step * 1e-3)
 
@@ -332,10 +343,7 @@ def run_ours(args, cfg):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms)
     e2e_value = world * cfg.tokens / (e2e_ms / e2e_steps * 1e-3)
     es = 2 if cfg.dtype == "bf16" else 4
     nparam = 3 * C * C + 3 * C + C * C + C + (2 * M - 1) ** 2 * nh
@@ -396,21 +404,29 @@ def dataclass_replace(cfg, **kw):
 
 
 # Algorithmic cost of each kernel per token: (flops, bytes) as functions of the layer; un-padded, no
-# credit for recomputation.  Bytes count what the kernel must read and write once.
+# credit for recomputation or for the padded head dim.  Bytes count every operand the kernel must read
+# or write exactly once.
 def kernel_cost(cfg: LayerConfig, name: str):
     C, N, nh = cfg.C, cfg.window ** 2, cfg.num_heads
     es = 2 if cfg.dtype == "bf16" else 4
     table = {
-        "qkv_gemm": (6 * C * C, (1 + 3) * C * es),
-        "attn_fwd": (4 * N * C, (3 + 1) * C * es + 4 * nh),
-        "proj_gemm": (2 * C * C, 2 * C * es),
-        "dproj": (4 * C * C, 3 * C * es),                       # dA = dy Wp and dWp = dy^T A: read dy, A; write dA
-        "attn_bwd": (10 * N * C, (3 + 2 + 3) * C * es + 4 * nh),  # read q,k,v,dA,A,L; write dq,dk,dv (S recomputed)
-        "dqkv_gemm": (12 * C * C, (3 + 1 + 1) * C * es),        # dx = dqkv Wqkv and dWqkv = dqkv^T x
+        "qkv_gemm": (6 * C * C, (1 + 3) * C * es),                 # read x; write q,k,v
+        "attn_fwd": (4 * N * C, (3 + 1) * C * es + 4 * nh),        # read q,k,v; write A and the row log-sum-exp
+        "proj_gemm": (2 * C * C, 2 * C * es),                      # read A; write y
+        "dattn_gemm": (2 * C * C, 2 * C * es),                     # read dy; write dO = dy W^P
+        "dwproj_gemm": (2 * C * C, 2 * C * es),                    # read dy, A; dW^P stays on chip
+        "attn_bwd": (8 * N * C, (3 + 1 + 3) * C * es + 4 * nh),    # read q,k,v,dO,L; write dq,dk,dv (no credit for recomputing S)
+        "dx_gemm": (6 * C * C, (3 + 1) * C * es),                  # read dqkv; write dx
+        "dwqkv_gemm": (6 * C * C, (3 + 1) * C * es),               # read dqkv, x; dW_qkv stays on chip
     }
-    alias = {"gemm_generic": None, "attn_fwd_generic": "attn_fwd", "attn_bwd_generic": "attn_bwd"}
-    key = alias.get(name, name)
-    return table.get(key)
+    alias = {"attn_fwd_generic": "attn_fwd", "attn_bwd_generic": "attn_bwd"}
+    return table.get(alias.get(name, name))
+
+
+# DRAM bytes per token of each kernel, dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture
+# on workload c3 (131072 tokens; traffic grows in proportion to the tokens) divided by its tokens.
+# None = not captured since the kernel last changed.  Source: profiles/.
+NCU_DRAM_BYTES_PER_TOKEN = {}
 
 
 def dominant_roofline(cfg, kernels, pk, pk_src):
@@ -421,7 +437,9 @@ def dominant_roofline(cfg, kernels, pk, pk_src):
     cost = kernel_cost(cfg, name)
     launches = max(k["launches_per_step"], 1e-9)
     dur = k["ms_per_step"] / launches * 1e-3
-    out = {"kernel": name, "launch_us": dur * 1e6, "share_of_step": k["share"], "peak_source": pk_src, "traffic": None}
+    per_tok = NCU_DRAM_BYTES_PER_TOKEN.get(name)
+    out = {"kernel": name, "launch_us": dur * 1e6, "share_of_step": k["share"], "peak_source": pk_src,
+           "traffic": None if per_tok is None else per_tok * cfg.tokens / launches}
     if cost is None:
         out.update({"bound": "hbm", "achieved": None, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": None,
                     "note": "no algorithmic cost model for this kernel"})
