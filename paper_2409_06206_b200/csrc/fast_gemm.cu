@@ -106,12 +106,26 @@ struct RingPos {
   }
 };
 
-// One thread of a loader set (64 threads): tile rows lw + 8k (lw = 0..7) and the 16-byte chunk `pp` of the
-// 128-byte atom row, copied as two 8-byte pieces because the caller's rows are only 8-byte aligned.
-// Consecutive lanes take consecutive chunks of the same row, so one copy instruction reads four rows
-// of 128 contiguous bytes.  Tile row r = lw + 8k has (r & 7) == lw: the swizzled destination is
-// dst0 + 1024 k.
+// One thread of a loader set (64 threads): the 8-byte piece `pc` (0..15) of the 128-byte atom row, in tile
+// rows rq + 4k (rq = 0..3).  Sixteen consecutive lanes cover one whole atom row: a copy instruction
+// reads two runs of 128 contiguous bytes and writes two full rows of shared memory (no bank
+// conflicts).  (r & 7) alternates between rq (k even) and rq + 4 (k odd), hence two swizzled bases;
+// the destination of row rq + 4k is base + 512 k.
 struct LoaderLane {
+  int rq, pc;
+  uint32_t dst_e, dst_o;
+  __device__ __forceinline__ void init(int ts) {
+    rq = ts >> 4;
+    pc = ts & 15;
+    dst_e = sw128_offset(rq, pc * 4);
+    dst_o = sw128_offset(rq + 4, pc * 4) - 4 * 128;
+  }
+  __device__ __forceinline__ uint32_t dst(int k) const { return (uint32_t)(k * 512) + ((k & 1) ? dst_o : dst_e); }
+};
+
+// Lane mapping of gr_kernel's copy-fed operand: rows lw + 8k, 16-byte chunk pp of the atom row (two
+// 8-byte pieces); a copy instruction reads four rows of 128 contiguous bytes.
+struct LoaderLane4 {
   int lw, pp;
   uint32_t dst0;
   __device__ __forceinline__ void init(int ts) {
@@ -196,8 +210,9 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
     int g = set;                                 // ring step = tile iteration * NA + atom
     int it = 0;
     for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
-      // the two windows of the pair: cyclic shift + partition are this address arithmetic
-      const char* col0[2];
+      // the two windows of the pair: cyclic shift + partition are this address arithmetic.  Tile row
+      // r = 64*half + 8*a + lw holds slot (a, lw) of window `half`; this thread owns lw = rq and rq + 4.
+      const char* col0[2][2];
       int i0[2];
       bool wv[2];
 #pragma unroll
@@ -206,28 +221,31 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
         wv[half] = win < (int)u.n_windows;
         const int b = win / u.nW, w = win - b * u.nW;
         const int wi = w / u.nWw, wj = w - wi * u.nWw;
-        int j = wj * 8 + ll.lw + u.s;
-        if (j >= u.W) j -= u.W;
         i0[half] = wi * 8 + u.s;
-        col0[half] = srcA + ((long long)b * u.H * u.W + j) * row_bytes + ll.pp * 16;
+#pragma unroll
+        for (int v = 0; v < 2; ++v) {
+          int j = wj * 8 + ll.rq + 4 * v + u.s;
+          if (j >= u.W) j -= u.W;
+          col0[half][v] = srcA + ((long long)b * u.H * u.W + j) * row_bytes + ll.pc * 8;
+        }
       }
       bool ok = true;
       for (; g < (it + 1) * NA; g += kSets) {
         const int atom = g - it * NA;
         if (!wait_bar_warp(&empty[rp.slot], rp.ph ^ 1, &abort_s, L.err)) { ok = false; break; }
-        const uint32_t dst = ringA + rp.slot * kAtomBytes + ll.dst0;
-        const int colb = atom * 128 + ll.pp * 16;          // byte offset inside a source row
-        const bool v0 = colb < u.kvalid * 2, v1 = colb + 8 < u.kvalid * 2;
+        const uint32_t dst = ringA + rp.slot * kAtomBytes;
+        const bool cv = atom * 128 + ll.pc * 8 < u.kvalid * 2;      // inside the valid columns of a source row
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
+          const bool v = wv[half] && cv;
 #pragma unroll
           for (int a8 = 0; a8 < 8; ++a8) {
             int i = i0[half] + a8;
             if (i >= u.H) i -= u.H;
-            const char* src = col0[half] + i * line_bytes + atom * 128;
-            const uint32_t d = dst + (8 * half + a8) * 1024;
-            cp_async8(d, wv[half] && v0 ? src : srcA, wv[half] && v0);
-            cp_async8(d + 8, wv[half] && v1 ? src + 8 : srcA, wv[half] && v1);
+            const long long off = i * line_bytes + atom * 128;
+            const int k = 16 * half + 2 * a8;
+            cp_async8(dst + ll.dst(k), v ? col0[half][0] + off : srcA, v);
+            cp_async8(dst + ll.dst(k + 1), v ? col0[half][1] + off : srcA, v);
           }
         }
         cp_async_commit();
@@ -529,7 +547,7 @@ __global__ void __launch_bounds__(kThreads, 1) gr_kernel(const __grid_constant__
     // 8-byte pieces, and the step is published as soon as the set's own copies have landed.
     const int set = (warp - kEpiWarps - 1) >> 1;
     const int ts = ((warp - kEpiWarps - 1) & 1) * 32 + lane;
-    LoaderLane ll;
+    LoaderLane4 ll;
     ll.init(ts);
     const int copy_base = L.tma_is_L ? 2 * 8192 : 0;                       // copy-fed operand inside a stage
     const int copy_atoms = L.tma_is_L ? ratoms : 2;
