@@ -377,7 +377,7 @@ def run_ours(args, cfg):
 
     cpu = None
     if world == 1 and not args.no_cpu:
-        images = 8
+        images = min(cfg.B, 40)                     # about 10-15 s of CPU work at C = 180
         v, dt, tokens = time_oracle(cfg, images)
         cpu = {"value": v, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
                "sample": "%d of %d images of %s (%d tokens) in %.1f s, numpy float64 fwd+bwd" % (
@@ -426,7 +426,7 @@ def kernel_cost(cfg: LayerConfig, name: str):
 # DRAM bytes per token of each kernel, dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture
 # on workload c3 (131072 tokens; traffic grows in proportion to the tokens) divided by its tokens.
 # None = not captured since the kernel last changed.  Source: profiles/.
-NCU_DRAM_BYTES_PER_TOKEN = {}
+NCU_DRAM_BYTES_PER_TOKEN = {"attn_bwd": 316.74e6 / 131072}   # profiles/attn_bwd_c3_ncu.md
 
 
 def dominant_roofline(cfg, kernels, pk, pk_src):
