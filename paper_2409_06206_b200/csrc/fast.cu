@@ -205,27 +205,54 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
   int rc = launch_prep(jobs, nj, st);
   if (rc) return rc;
 
-  GWLaunch gw{};
-  gw.err = err;
-  for (int i = 0; i < nu; ++i) {
-    const Unit& u = units[i];
-    GWUnit& w = gw.u[i];
-    w.A = (const bf*)x; w.lda = p.C; w.kvalid = p.C;
-    w.H = p.H; w.W = p.W; w.s = p.gs[u.g]; w.nW = p.nW; w.nWw = p.nWw; w.n_windows = geo.n_windows;
-    w.Bimg = (const unsigned char*)sc + fs.img[i];
-    w.bias = (const float*)(sc + fs.bias[i]);
-    w.out = qkv + geo.qkv_off[u.g] + (long long)(u.h0 - p.gh0[u.g]) * 3 * 64 * p.dp;
-    w.win_stride = (long long)p.gh[u.g] * 3 * 64 * p.dp;
-    w.nchunks = u.nheads; w.cw = 3 * p.dp; w.q_every3 = 1;
-    w.qscale = 1.4426950408889634f / sqrtf((float)p.d);   // d^-1/2 and log2(e): the attention kernels work in the log2 domain
-  }
-  if ((rc = launch_gw(gw, nu, p.Cp, p.dp, st, "qkv_gemm"))) return rc;
+  const float qscale = 1.4426950408889634f / sqrtf((float)p.d);   // d^-1/2 and log2(e): attention works in the log2 domain
+  int maxh = 0;
+  for (int i = 0; i < nu; ++i) maxh = units[i].nheads > maxh ? units[i].nheads : maxh;
+  if ((p.flags & GSWA_FLAG_FUSED_FWD) && fw_smem_bytes(p.Cp, p.dp, maxh, nullptr) != 0) {
+    // fused (opt-in): projection and attention of a window pair in one CTA; q,k,v reach HBM only when
+    // the backward pass will need them.  Measured slower than the two kernels below at C = 180 (the
+    // twelve attention warps that fit beside the GEMM's shared memory cannot hide their own latency).
+    FWLaunch fw{};
+    fw.geo = geo; fw.table = (const bf*)table; fw.A = A; fw.err = err;
+    for (int i = 0; i < nu; ++i) {
+      const Unit& u = units[i];
+      FWUnit& w = fw.u[i];
+      const int hl0 = u.h0 - p.gh0[u.g];
+      w.X = (const bf*)x; w.lda = p.C; w.kvalid = p.C;
+      w.H = p.H; w.W = p.W; w.s = p.gs[u.g]; w.nW = p.nW; w.nWw = p.nWw; w.n_windows = geo.n_windows;
+      w.Bimg = (const unsigned char*)sc + fs.img[i];
+      w.bias = (const float*)(sc + fs.bias[i]);
+      w.qscale = qscale;
+      w.h0 = u.h0; w.nheads = u.nheads;
+      w.qkv_out = want_L ? qkv + geo.qkv_off[u.g] + (long long)hl0 * 3 * 64 * p.dp : nullptr;
+      w.qkv_wstride = (long long)p.gh[u.g] * 3 * 64 * p.dp;
+      w.lt = want_L ? Lt + geo.l_off[u.g] + (long long)hl0 * 64 : nullptr;
+      w.l_wstride = (long long)p.gh[u.g] * 64;
+    }
+    if ((rc = launch_fw(fw, nu, p.Cp, p.dp, st))) return rc;
+  } else {
+    GWLaunch gw{};
+    gw.err = err;
+    for (int i = 0; i < nu; ++i) {
+      const Unit& u = units[i];
+      GWUnit& w = gw.u[i];
+      w.A = (const bf*)x; w.lda = p.C; w.kvalid = p.C;
+      w.H = p.H; w.W = p.W; w.s = p.gs[u.g]; w.nW = p.nW; w.nWw = p.nWw; w.n_windows = geo.n_windows;
+      w.Bimg = (const unsigned char*)sc + fs.img[i];
+      w.bias = (const float*)(sc + fs.bias[i]);
+      w.out = qkv + geo.qkv_off[u.g] + (long long)(u.h0 - p.gh0[u.g]) * 3 * 64 * p.dp;
+      w.win_stride = (long long)p.gh[u.g] * 3 * 64 * p.dp;
+      w.nchunks = u.nheads; w.cw = 3 * p.dp; w.q_every3 = 1;
+      w.qscale = qscale;
+    }
+    if ((rc = launch_gw(gw, nu, p.Cp, p.dp, st, "qkv_gemm"))) return rc;
 
-  AttnLaunch al{};
-  attn_units(p, geo, units, nu, &al);
-  al.qkv = qkv; al.table = (const bf*)table; al.A = A; al.Lt = want_L ? Lt : nullptr;
-  al.scale = 1.0f / sqrtf((float)p.d);
-  if ((rc = launch_attn_fwd(al, st))) return rc;
+    AttnLaunch al{};
+    attn_units(p, geo, units, nu, &al);
+    al.qkv = qkv; al.table = (const bf*)table; al.A = A; al.Lt = want_L ? Lt : nullptr;
+    al.scale = 1.0f / sqrtf((float)p.d);
+    if ((rc = launch_attn_fwd(al, st))) return rc;
+  }
 
   GTLaunch gt{};
   if ((rc = make_tmap(&gt.tmA, A, p.T, p.Ap, 128))) return rc;

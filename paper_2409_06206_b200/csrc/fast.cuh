@@ -109,6 +109,34 @@ struct GRLaunch {
 };
 
 int launch_gw(const GWLaunch& L, int nunits, int Cp, int dp, cudaStream_t st, const char* name);
+
+// ---- fused forward: QKV projection of a window pair on the tensor core, its q,k,v tiles handed to the
+// attention warps of the same CTA through shared memory (and, for training, shipped to `qkv_out`).
+struct FWUnit {
+  const __nv_bfloat16* X;      // x, pitch lda elements, kvalid valid columns
+  int lda, kvalid;
+  int H, W, s, nW, nWw;
+  long long n_windows;
+  const unsigned char* Bimg;   // QKV weight image of this unit's heads: [KP/64 atoms][NT rows][128 B]
+  const float* bias;           // [NT] or nullptr
+  float qscale;                // d^-1/2 * log2(e), applied to the q blocks
+  int h0, nheads;              // first head (global index), heads in this unit
+  __nv_bfloat16* qkv_out;      // tile image of this unit's first block in window 0, or nullptr (inference)
+  long long qkv_wstride;       // elements between consecutive windows
+  float* lt;                   // row log-sum-exp tiles of this unit in window 0, or nullptr
+  long long l_wstride;
+};
+struct FWLaunch {
+  FWUnit u[kMaxUnits];
+  FastGeom geo;
+  const __nv_bfloat16* table;  // [(2M-1)^2, nh]
+  __nv_bfloat16* A;            // [T, Ap] out
+  int* err;
+  int nslots;                  // ring slots of 16 KB (set by launch_fw)
+};
+// Shared memory the fused kernel needs for units of at most `maxheads` heads (0 if it cannot run).
+size_t fw_smem_bytes(int Cp, int dp, int maxheads, int* nslots);
+int launch_fw(const FWLaunch& L, int nunits, int Cp, int dp, cudaStream_t st);
 int launch_gt(const GTLaunch& L, int nsplits, cudaStream_t st, const char* name);
 int launch_gr(const GRLaunch& L, cudaStream_t st, const char* name);
 // Tensor map of a padded token-major bf16 buffer [rows, cols]: box 64 columns x box_rows rows, 128-byte swizzle.

@@ -11,205 +11,17 @@
 // The backward pass keeps only the row log-sum-exp from the forward pass: P = exp(S - L) is rebuilt
 // per window, D = rowsum(P * dP) replaces the usual dO.O term, and P / dS cross from the
 // query-major phase (dQ) to the key-major phase (dK, dV) through shared memory.
-#include "fast.cuh"
-#include "gswa_index.cuh"
+#include "attn_core.cuh"
 
 namespace gswa {
+using namespace attn;
 namespace {
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-__device__ __forceinline__ void ldsm_x4(uint32_t* r, uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-               : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t* r, uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-               : "r"(addr));
-}
-__device__ __forceinline__ void mma16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-
-constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
-
-__device__ __forceinline__ float ex2(float x) {          // 2^x, one MUFU instruction; 2^-inf = 0
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ void stsm_x4(uint32_t addr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3) {
-  asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
-               : "memory");
-}
-__device__ __forceinline__ void stsm_x2(uint32_t addr, uint32_t r0, uint32_t r1) {
-  asm volatile("stmatrix.sync.aligned.m8n8.x2.shared.b16 [%0], {%1,%2};" ::"r"(addr), "r"(r0), "r"(r1) : "memory");
-}
-
-// [64][64] bf16 matrices (P, dS): 128-byte rows, chunk ^= row & 7.
-__device__ __forceinline__ uint32_t sq_off(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
-
-// Tiles arrive from global memory already in their shared-memory image (tile_off): a linear copy.
-template <int DP>
-__device__ __forceinline__ void load_tiles(unsigned char* dst, const __nv_bfloat16* src, int nblocks, int tid, int nt) {
-  const int nchunks = nblocks * 64 * (DP / 8);
-  const uint32_t d0 = smem_u32(dst);
-  for (int ci = tid; ci < nchunks; ci += nt)
-    cp_async16(d0 + ci * 16, reinterpret_cast<const unsigned char*>(src) + (size_t)ci * 16);
-}
-
-// S (16 rows x 64 keys) = Q K^T for the warp's rows; returns accumulators in s[8][4].
-template <int DP>
-__device__ __forceinline__ void qk_scores(float (*s)[4], uint32_t q_base, uint32_t k_base, int r0, int lane) {
-#pragma unroll
-  for (int j = 0; j < 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
-#pragma unroll
-  for (int kk = 0; kk < DP / 16; ++kk) {
-    uint32_t a[4];
-    ldsm_x4(a, q_base + tile_off<DP>(r0 + (lane & 15), 2 * kk + (lane >> 4)));
-#pragma unroll
-    for (int jp = 0; jp < 4; ++jp) {
-      uint32_t b[4];
-      ldsm_x4(b, k_base + tile_off<DP>(16 * jp + (lane & 7) + ((lane >> 4) << 3), 2 * kk + ((lane >> 3) & 1)));
-      mma16816(s[2 * jp], a, b[0], b[1]);
-      mma16816(s[2 * jp + 1], a, b[2], b[3]);
-    }
-  }
-}
-
-// acc (16 x DP) += A(16 x 64, from packed register fragments of `pf`) * B(64 x DP) with B read
-// transposed from a [64][DP] tile (rows = contraction index).
-template <int DP>
-__device__ __forceinline__ void regs_times_tile(float (*acc)[4], const float (*pf)[4], uint32_t b_base, int lane) {
-#pragma unroll
-  for (int kk = 0; kk < 4; ++kk) {
-    uint32_t a[4];
-    a[0] = pack2(pf[2 * kk][0], pf[2 * kk][1]);
-    a[1] = pack2(pf[2 * kk][2], pf[2 * kk][3]);
-    a[2] = pack2(pf[2 * kk + 1][0], pf[2 * kk + 1][1]);
-    a[3] = pack2(pf[2 * kk + 1][2], pf[2 * kk + 1][3]);
-#pragma unroll
-    for (int jn = 0; jn < DP / 16; ++jn) {
-      uint32_t b[4];
-      ldsm_x4_t(b, b_base + tile_off<DP>(16 * kk + (lane & 7) + (((lane >> 3) & 1) << 3), 2 * jn + (lane >> 4)));
-      mma16816(acc[2 * jn], a, b[0], b[1]);
-      mma16816(acc[2 * jn + 1], a, b[2], b[3]);
-    }
-  }
-}
-
-__device__ __forceinline__ void set_word(uint4& v, int i, uint32_t w) {
-  if (i == 0) v.x = w; else if (i == 1) v.y = w; else if (i == 2) v.z = w; else v.w = w;
-}
-
-// Writes a warp's 16 x DP accumulator tile (rows gq, gq+8 of the mma fragment) to rows of a padded
-// token-major buffer: the tile is first laid out in the warp's 16 x DP staging block (stmatrix), then
-// every lane moves 16 bytes per row so that one store instruction covers whole 2*DP-byte row pieces.
-// `row0` / `row1` are the global addresses of the lane's two rows (fragment rows gq and gq + 8).
-template <int DP>
-__device__ __forceinline__ void store_tile(unsigned char* stg, const float (*acc)[4], float scale, unsigned char* row0,
-                                           unsigned char* row1, int lane, int ones_col) {
-  const uint32_t sa = smem_u32(stg);
-  const int m = lane >> 3;
-#pragma unroll
-  for (int jn = 0; jn < DP / 8; jn += 2) {
-    const int row = (m & 1) * 8 + (lane & 7), chunk = jn + (m >> 1);
-    stsm_x4(sa + tile_off<DP>(row, chunk), pack2(acc[jn][0] * scale, acc[jn][1] * scale),
-            pack2(acc[jn][2] * scale, acc[jn][3] * scale), pack2(acc[jn + 1][0] * scale, acc[jn + 1][1] * scale),
-            pack2(acc[jn + 1][2] * scale, acc[jn + 1][3] * scale));
-  }
-  __syncwarp();
-  if constexpr (DP == 32) {
-    const int gq = lane >> 2, t = lane & 3;
-    uint4 v0 = *reinterpret_cast<const uint4*>(stg + tile_off<DP>(gq, t));
-    uint4 v1 = *reinterpret_cast<const uint4*>(stg + tile_off<DP>(gq + 8, t));
-    if (ones_col >= 0 && (ones_col >> 3) == t) {
-      set_word(v0, (ones_col & 7) >> 1, 0x00003F80u);        // (1.0, 0.0)
-      set_word(v1, (ones_col & 7) >> 1, 0x00003F80u);
-    }
-    *reinterpret_cast<uint4*>(row0 + t * 16) = v0;
-    *reinterpret_cast<uint4*>(row1 + t * 16) = v1;
-  } else {
-    // DP == 16: 16 rows x 2 chunks, one chunk per lane; the lane's row pointer comes from a neighbour
-    const int r = lane >> 1, c = lane & 1;
-    uint4 v = *reinterpret_cast<const uint4*>(stg + tile_off<DP>(r, c));
-    if (ones_col >= 0 && (ones_col >> 3) == c) set_word(v, (ones_col & 7) >> 1, 0x00003F80u);
-    // row pointers live in lanes with gq == r (rows 0..7: row0 of lane 4r) or gq == r - 8 (row1 of lane 4(r-8))
-    const unsigned long long a0 = __shfl_sync(0xffffffffu, (unsigned long long)row0, (r & 7) * 4);
-    const unsigned long long a1 = __shfl_sync(0xffffffffu, (unsigned long long)row1, (r & 7) * 4);
-    *reinterpret_cast<uint4*>((r < 8 ? a0 : a1) + c * 16) = v;
-  }
-  __syncwarp();
-}
-
-struct WinCtx {
-  int b, wi, wj;
-  bool masked;
-};
-
-__device__ __forceinline__ WinCtx window_setup(const FastGeom& g, int s, long long win, int* tok, unsigned char* reg,
-                                               int tid) {
-  WinCtx c;
-  c.b = (int)(win / g.nW);
-  const int w = (int)(win % g.nW);
-  c.wi = w / g.nWw;
-  c.wj = w % g.nWw;
-  c.masked = s > 0 && (c.wi == g.nWh - 1 || c.wj == g.nWw - 1);
-  if (tid < 64) {
-    int i, j, r;
-    slot_to_token(g.H, g.W, 8, s, w, tid, &i, &j, &r);
-    tok[tid] = (c.b * g.H + i) * g.W + j;
-    reg[tid] = (unsigned char)r;
-  }
-  return c;
-}
-
-// Adds the relative-position bias and applies the mask (scores are in the log2 domain throughout).
-__device__ __forceinline__ void bias_and_mask(float (*s)[4], const float* tab, const unsigned char* reg, bool masked,
-                                              int p0, int t) {
-  const int pa0 = p0 >> 3, pc0 = p0 & 7;   // rows p0 and p0 + 8: same column in the window, next row
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int pa = pa0 + (e >> 1), qc = 2 * t + (e & 1);
-      const int rel = (pa - j + 7) * 15 + (pc0 - qc + 7);
-      s[j][e] += tab[rel];                  // q and the table are already scaled by log2(e)
-    }
-  }
-  if (masked) {
-    const unsigned char r0 = reg[p0], r1 = reg[p0 + 8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const unsigned char q0 = reg[8 * j + 2 * t], q1 = reg[8 * j + 2 * t + 1];
-      if (q0 != r0) s[j][0] = -INFINITY;
-      if (q1 != r0) s[j][1] = -INFINITY;
-      if (q0 != r1) s[j][2] = -INFINITY;
-      if (q1 != r1) s[j][3] = -INFINITY;
-    }
-  }
-}
 
 // ------------------------------------------------------------------------------------------
 // forward: persistent CTAs stride over the windows of a unit; 4 warps per head, 16 query rows per
 // warp.  The q,k,v tiles of the next window are copied into the second buffer while the current
 // window is being computed.
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ void cp_async_wait_1() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-
 template <int DP>
 __global__ void __launch_bounds__(384, 2) attn_fwd_kernel(const __grid_constant__ AttnLaunch L) {
   const AttnUnit& u = L.u[blockIdx.y];
@@ -248,57 +60,9 @@ __global__ void __launch_bounds__(384, 2) attn_fwd_kernel(const __grid_constant_
 
     unsigned char* tiles = sm + (size_t)buf * tile_bytes;
     const uint32_t q_base = smem_u32(tiles + (size_t)(hl * 3 + 0) * 64 * DP * 2);
-    const uint32_t k_base = q_base + 64 * DP * 2, v_base = k_base + 64 * DP * 2;
-    float s[8][4];
-    qk_scores<DP>(s, q_base, k_base, r0, lane);
-    bias_and_mask(s, tab + hl * 225, reg, wc.masked, p0, t);
-
-    float m0 = -INFINITY, m1 = -INFINITY;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      m0 = fmaxf(m0, fmaxf(s[j][0], s[j][1]));
-      m1 = fmaxf(m1, fmaxf(s[j][2], s[j][3]));
-    }
-    m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1));
-    m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
-    m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1));
-    m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
-    float sum0 = 0.f, sum1 = 0.f;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      s[j][0] = ex2(s[j][0] - m0);
-      s[j][1] = ex2(s[j][1] - m0);
-      s[j][2] = ex2(s[j][2] - m1);
-      s[j][3] = ex2(s[j][3] - m1);
-      sum0 += s[j][0] + s[j][1];
-      sum1 += s[j][2] + s[j][3];
-    }
-    sum0 += __shfl_xor_sync(0xffffffffu, sum0, 1);
-    sum0 += __shfl_xor_sync(0xffffffffu, sum0, 2);
-    sum1 += __shfl_xor_sync(0xffffffffu, sum1, 1);
-    sum1 += __shfl_xor_sync(0xffffffffu, sum1, 2);
-
-    float o[DP / 8][4];
-#pragma unroll
-    for (int j = 0; j < DP / 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
-    regs_times_tile<DP>(o, s, v_base, lane);
-
-    // rows of the padded attention output: DP columns per head, pad columns are exact zeros because
-    // the pad columns of v are; column d of head 0 is set to one (bias-gradient column, see fast.cuh)
-    const float inv0 = 1.f / sum0, inv1 = 1.f / sum1;
-#pragma unroll
-    for (int jn = 0; jn < DP / 8; ++jn) {
-      o[jn][0] *= inv0; o[jn][1] *= inv0; o[jn][2] *= inv1; o[jn][3] *= inv1;
-    }
-    const int Ap = g.nh * DP;
-    store_tile<DP>(ostg, o, 1.f, reinterpret_cast<unsigned char*>(L.A + (long long)tok[p0] * Ap + h * DP),
-                   reinterpret_cast<unsigned char*>(L.A + (long long)tok[p0 + 8] * Ap + h * DP), lane,
-                   (h == 0 && g.d < DP) ? g.d : -1);
-    if (L.Lt != nullptr && t == 0) {
-      float* lt = L.Lt + u.l_off + win * u.l_wstride + hl * 64;
-      lt[p0] = m0 * kLn2 + logf(sum0);
-      lt[p0 + 8] = m1 * kLn2 + logf(sum1);
-    }
+    fwd_window<DP>(q_base, q_base + 64 * DP * 2, q_base + 2 * 64 * DP * 2, tab + hl * 225, tok, reg, wc.masked, r0, lane,
+                   ostg, L.A, g.nh * DP, h, g.d,
+                   L.Lt != nullptr ? L.Lt + u.l_off + win * u.l_wstride + hl * 64 : nullptr);
     __syncthreads();   // every warp is done with this buffer before the next iteration refills it
   }
   cp_async_wait_all();

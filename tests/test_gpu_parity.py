@@ -88,6 +88,17 @@ def test_generic_kernels_forced(cfg):
     assert_close(got, ref, cfg.dtype)
 
 
+@pytest.mark.parametrize("cfg", [SWEEP[7], SWEEP[8], SWEEP[9], SWEEP[11]], ids=["c60", "c180", "uneven-groups", "two-heads"])
+def test_fused_forward_kernel(cfg):
+    """The opt-in kernel that fuses the QKV projection with the forward attention (training and inference mode)."""
+    inp = make_inputs(cfg)
+    got = run_gpu(cfg, inp, flags=gb.FLAG_FUSED_FWD)
+    ref = run_oracle(cfg, inp)
+    assert_close(got, ref, cfg.dtype)
+    inf = run_gpu(cfg, inp, flags=gb.FLAG_FUSED_FWD, inference=True)
+    assert rel_err(inf["y"], got["y"]) == 0.0
+
+
 def test_null_biases_inference_mode_and_accumulate():
     import torch
     cfg = dataclasses.replace(SWEEP[7], bias_std=0.0)
