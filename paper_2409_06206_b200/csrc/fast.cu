@@ -319,11 +319,12 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
     // dW^P = dy^T A (A fetched by TMA); db^P rides on the ones column of A when the head dim is padded
     GRLaunch gr{};
     if ((rc = make_tmap(&gr.tm, A, p.T, p.Ap, 64))) return rc;
-    gr.tma_is_L = 0; gr.use_tma = 1; gr.Q = A; gr.qcols = p.Ap;
+    gr.tma_is_L = 0;
     gr.P = (const bf*)dy; gr.ldp = p.C; gr.pvalid = p.C;
     gr.Ap = p.Ap; gr.dp = p.dp; gr.d = p.d; gr.C = p.C; gr.M = p.C; gr.rows = p.T;
     gr.NP = (int)align_up((size_t)p.Ap, 64);
-    const int mblocks = (p.C + 127) / 128;
+    gr.mbpc = 1;                                   // two M blocks per CTA measured slower here (fewer TMA stages)
+    const int mblocks = ((p.C + 127) / 128 + gr.mbpc - 1) / gr.mbpc;
     long long ns = sms / mblocks, cap = (p.T + 63) / 64;
     gr.nsplit = (int)(ns < cap ? (ns < 1 ? 1 : ns) : cap);
     gr.out = dw_proj ? dw_proj : dummy; gr.colsum = p.d < p.dp ? db_proj : nullptr; gr.err = err;
@@ -352,11 +353,12 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
     // dW_qkv = dqkv^T x (dqkv fetched by TMA); db_qkv from a column of ones appended to x
     GRLaunch gr{};
     if ((rc = make_tmap(&gr.tm, dqkv, p.T, 3 * p.Ap, 64))) return rc;
-    gr.tma_is_L = 1; gr.use_tma = 1; gr.Q = dqkv; gr.qcols = 3 * p.Ap;
+    gr.tma_is_L = 1;
     gr.P = (const bf*)x; gr.ldp = p.C; gr.pvalid = p.C;
     gr.Ap = p.Ap; gr.dp = p.dp; gr.d = p.d; gr.C = p.C; gr.M = 3 * p.Ap; gr.rows = p.T;
     gr.NP = np_cols(p.C);
-    const int mblocks = (3 * p.Ap + 127) / 128;
+    gr.mbpc = 2 * gr.NP <= 512 ? 2 : 1;            // x is copied once for two M blocks of dqkv
+    const int mblocks = ((3 * p.Ap + 127) / 128 + gr.mbpc - 1) / gr.mbpc;
     long long ns = sms / mblocks, cap = (p.T + 63) / 64;
     gr.nsplit = (int)(ns < cap ? (ns < 1 ? 1 : ns) : cap);
     gr.out = dw_qkv ? dw_qkv : dummy; gr.colsum = db_qkv; gr.err = err;

@@ -91,9 +91,6 @@ struct GTLaunch {
 // Padded indices (kind, head, c) map to kind*C + head*d + c; c >= d is dropped.
 struct GRLaunch {
   CUtensorMap tm;
-  int use_tma;                 // 1: padded operand through TMA; 0: through 16-byte asynchronous copies
-  const __nv_bfloat16* Q;      // the padded operand [rows, qcols]
-  int qcols;
   int tma_is_L;
   const __nv_bfloat16* P;      // the copy-fed operand, [rows, ldp] with pvalid valid columns
   int ldp, pvalid;
@@ -102,7 +99,8 @@ struct GRLaunch {
   long long rows;
   int NP;                      // accumulator columns (multiple of 64)
   int nsplit;                  // token splits
-  int nstages;                 // ring depth (set by launch_gr)
+  int mbpc;                    // M blocks of 128 handled by one CTA (1 or 2)
+  int nstages;                 // depth of the TMA ring (set by launch_gr)
   float* out;                  // float, accumulated with atomics: [3C, C] or [C, C]
   float* colsum;               // or nullptr: dB[m] = sum_t L[t, m]
   int* err;

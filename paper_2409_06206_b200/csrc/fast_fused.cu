@@ -273,7 +273,8 @@ size_t fw_smem_bytes(int Cp, int dp, int maxheads, int* nslots) {
   const size_t fixed = 1024 + NT * Cp * 2 + (size_t)maxheads * 3 * 64 * dp * 2 + NT * 4 + (size_t)maxheads * 225 * 4 + 64 * 4 + 64 +
                        16 + (size_t)kAttnWarps * 16 * dp * 2 + 64;
   const size_t budget = 224 * 1024;
-  if (fixed + (size_t)(Cp / 64) * 16384 > budget) return 0;
+  const int need = Cp / 64 > kSetsF ? Cp / 64 : kSetsF;      // a tile's atoms must fit, and no more loader sets than slots
+  if (fixed + (size_t)need * 16384 > budget) return 0;
   int s = (int)((budget - fixed) / 16384);
   if (s > 8) s = 8;
   if (nslots) *nslots = s;

@@ -369,108 +369,101 @@ __device__ __forceinline__ int unpad_index(int idx, int Ap, int dp, int d, int C
   return c < d ? kind * C + h * d + c : -1;
 }
 
-__global__ void __launch_bounds__(kThreads, 1) gr_kernel(const __grid_constant__ GRLaunch L) {
+__global__ void __launch_bounds__(kThreadsR, 1) gr_kernel(const __grid_constant__ GRLaunch L) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = align1024(smem_raw);
   const int NP = L.NP, ratoms = NP / 64;
-  const int stage_bytes = (2 + ratoms) * 8192;             // [L atom 0 | L atom 1 | R atoms], 64 tokens x 64 columns each
-  __shared__ uint64_t full[8], empty[8], done;
+  const int MB = L.mbpc, latoms = 2 * MB;                  // M blocks of 128 per CTA: the other operand is fetched once for all of them
+  // Two rings of 64-token stages: one for the padded operand that TMA fetches (deep, because those bytes
+  // come from HBM with microseconds of latency), one for the caller's tensor that the loader sets copy.
+  const int tma_atoms_all = L.tma_is_L ? latoms : ratoms;
+  const int copy_atoms = L.tma_is_L ? ratoms : latoms;
+  const int tbytes = tma_atoms_all * 8192, cbytes = copy_atoms * 8192;
+  const int ST = L.nstages, SC = kSets;
+  unsigned char* ringT = sm;
+  unsigned char* ringC = sm + (size_t)ST * tbytes;
+  __shared__ uint64_t fullT[8], emptyT[8], fullC[kSets], emptyC[kSets], done;
   __shared__ uint32_t tmem_s;
   __shared__ int abort_s;
-  const int S = L.nstages;                               // ring depth; S - 1 stages of loads stay in flight
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int mb = blockIdx.y;
+  const int mb = blockIdx.y * MB;                          // first M block of this CTA
   long long chunk = (L.rows + L.nsplit - 1) / L.nsplit;
   chunk = (chunk + 63) / 64 * 64;
   const long long t0 = (long long)blockIdx.x * chunk;
   const long long t1 = t0 + chunk < L.rows ? t0 + chunk : L.rows;
   if (t0 >= t1) return;
   const int nst = (int)((t1 - t0 + 63) / 64);
-  // atoms TMA brings per stage, and where they go
   const int tma_cols = L.tma_is_L ? L.M - mb * 128 : L.Ap;                 // valid columns of the TMA-fed operand here
-  const int tma_atoms = tma_cols >= (L.tma_is_L ? 128 : NP) ? (L.tma_is_L ? 2 : ratoms) : (tma_cols + 63) / 64;
-  const int tma_atoms_all = L.tma_is_L ? 2 : ratoms;
+  const int tma_atoms = (tma_cols + 63) / 64 < tma_atoms_all ? (tma_cols + 63) / 64 : tma_atoms_all;
 
   if (tid == 0) {
     abort_s = 0;
-    for (int i = 0; i < S; ++i) { mbar_init(&full[i], L.use_tma ? 3 : 2); mbar_init(&empty[i], 1); }   // two warps of a set (+ the TMA request)
+    for (int i = 0; i < 8; ++i) { mbar_init(&fullT[i], 1); mbar_init(&emptyT[i], 1); }
+    for (int i = 0; i < kSets; ++i) { mbar_init(&fullC[i], 2); mbar_init(&emptyC[i], 1); }
     mbar_init(&done, 1);
     mbar_init_fence();
   }
-  const uint32_t tcols = pow2_cols(NP);
+  const uint32_t tcols = pow2_cols(MB * NP);
   if (warp == kEpiWarps) tmem_alloc(&tmem_s, tcols);
   fence_before_sync();
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem = tmem_s;
 
-  if (warp > kEpiWarps) {
-    // ---------------- loaders: four sets of two warps; set q fills ring steps q, q+4, ...  Its leader
-    // asks TMA for the padded operand's 64-token boxes, all 64 threads copy the caller's rows in
-    // 8-byte pieces, and the step is published as soon as the set's own copies have landed.
-    const int set = (warp - kEpiWarps - 1) >> 1;
-    const int ts = ((warp - kEpiWarps - 1) & 1) * 32 + lane;
-    LoaderLane4 ll;
-    ll.init(ts);
-    const int copy_base = L.tma_is_L ? 2 * 8192 : 0;                       // copy-fed operand inside a stage
-    const int copy_atoms = L.tma_is_L ? ratoms : 2;
-    const int copy_col0 = L.tma_is_L ? 0 : mb * 128;                       // first column of the copy-fed operand here
-    // Pieces that never change (padding, the ones column, atoms TMA never touches) are written once per
-    // stage buffer, before the loop.
-    for (int sgi = set; sgi < S; sgi += kSets) {
-      unsigned char* base = sm + (size_t)sgi * stage_bytes;
-      for (int a = 0; a < copy_atoms; ++a)
-        for (int half = 0; half < 2; ++half) {
-          const int col = copy_col0 + a * 64 + ll.pp * 8 + half * 4;
-          if (col < L.pvalid) continue;
-          const uint2 val = make_uint2((L.tma_is_L && col == L.pvalid) ? 0x3F80u : 0u, 0u);
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            *reinterpret_cast<uint2*>(base + copy_base + a * 8192 + ll.dst0 + k * 1024 + half * 8) = val;
-        }
+  if (warp == kEpiWarps + 1) {
+    // ---------------- TMA producer: 64-token boxes of the padded operand, as far ahead as the ring allows.
+    // Atoms that lie wholly outside the tensor are never requested: they are zeroed once.
+    for (int sgi = 0; sgi < ST; ++sgi)
       for (int a = tma_atoms; a < tma_atoms_all; ++a) {
-        unsigned char* at = base + (L.tma_is_L ? 0 : 2 * 8192) + a * 8192;
-        for (int e = ts; e < 8192 / 16; e += 64) reinterpret_cast<uint4*>(at)[e] = make_uint4(0u, 0u, 0u, 0u);
+        unsigned char* at = ringT + (size_t)sgi * tbytes + a * 8192;
+        for (int e = lane; e < 8192 / 16; e += 32) reinterpret_cast<uint4*>(at)[e] = make_uint4(0u, 0u, 0u, 0u);
+      }
+    fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) {
+      RingPos rp;
+      rp.init(0, ST);
+      for (int s = 0; s < nst; ++s) {
+        if (!wait_bar(&emptyT[rp.slot], rp.ph ^ 1, &abort_s, L.err)) break;
+        const uint32_t dst = smem_u32(ringT + (size_t)rp.slot * tbytes);
+        mbar_arrive_expect_tx(&fullT[rp.slot], (uint32_t)tma_atoms * 8192u);
+        for (int a = 0; a < tma_atoms; ++a)
+          tma_load_2d(dst + a * 8192, &L.tm, (L.tma_is_L ? mb * 128 : 0) + a * 64, (int)(t0 + (long long)s * 64), &fullT[rp.slot]);
+        rp.advance(1, ST);
       }
     }
+  } else if (warp > kEpiWarps + 1) {
+    // ---------------- loader sets for the caller's tensor: set q fills copy-ring steps q, q+4, ... (slot q)
+    const int set = (warp - kEpiWarps - 2) >> 1;
+    const int ts = ((warp - kEpiWarps - 2) & 1) * 32 + lane;
+    LoaderLane4 ll;
+    ll.init(ts);
+    const int copy_col0 = L.tma_is_L ? 0 : mb * 128;                       // first column of the copy-fed operand here
+    unsigned char* base = ringC + (size_t)set * cbytes;
+    // Pieces that never change (padding, the ones column) are written once, before the loop.
+    for (int a = 0; a < copy_atoms; ++a)
+      for (int half = 0; half < 2; ++half) {
+        const int col = copy_col0 + a * 64 + ll.pp * 8 + half * 4;
+        if (col < L.pvalid) continue;
+        const uint2 val = make_uint2((L.tma_is_L && col == L.pvalid) ? 0x3F80u : 0u, 0u);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) *reinterpret_cast<uint2*>(base + a * 8192 + ll.dst0 + k * 1024 + half * 8) = val;
+      }
     const char* const srcP = reinterpret_cast<const char*>(L.P);
     const long long prow = (long long)L.ldp * 2;
-    RingPos rp;
-    rp.init(set, S);
-    for (int s = set; s < nst; s += kSets) {
-      if (!wait_bar_warp(&empty[rp.slot], rp.ph ^ 1, &abort_s, L.err)) break;
-      const uint32_t sS = smem_u32(sm + (size_t)rp.slot * stage_bytes);
+    const uint32_t sS = smem_u32(base);
+    int ph = 0;
+    for (int s = set; s < nst; s += kSets, ph ^= 1) {
+      if (!wait_bar_warp(&emptyC[set], ph ^ 1, &abort_s, L.err)) break;
       const long long tb = t0 + (long long)s * 64;
-      if (L.use_tma) {
-        if (ts == 0) {
-          // the TMA-fed operand; rows past the end of the tensor arrive as zeros
-          mbar_arrive_expect_tx(&full[rp.slot], (uint32_t)tma_atoms * 8192u);
-          for (int a = 0; a < tma_atoms; ++a)
-            tma_load_2d(sS + (L.tma_is_L ? 0 : 2 * 8192) + a * 8192, &L.tm, (L.tma_is_L ? mb * 128 : 0) + a * 64, (int)tb,
-                        &full[rp.slot]);
-        }
-      } else {
-        // the padded operand by 16-byte copies (its rows are 16-byte aligned)
-        const int qc0 = (L.tma_is_L ? mb * 128 : 0) + ll.pp * 8;
-        const char* q = reinterpret_cast<const char*>(L.Q) + ((tb + ll.lw) * (long long)L.qcols + qc0) * 2;
-        const uint32_t qd = sS + (L.tma_is_L ? 0 : 2 * 8192) + ll.dst0;
-        for (int a = 0; a < tma_atoms; ++a) {
-          const bool cv = qc0 + a * 64 < L.qcols;
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const bool v = cv && tb + ll.lw + 8 * k < L.rows;
-            cp_async16(qd + a * 8192 + k * 1024, v ? q + ((long long)k * 8 * L.qcols + a * 64) * 2 : (const char*)L.Q, v);
-          }
-        }
-      }
       const char* pp = srcP + (tb + ll.lw) * prow + (copy_col0 + ll.pp * 8) * 2;
       const bool whole = tb + 64 <= t1;
       for (int a = 0; a < copy_atoms; ++a) {
         const int col = copy_col0 + a * 64 + ll.pp * 8;
         const bool v0 = col < L.pvalid, v1 = col + 4 < L.pvalid;
         if (!v0) break;
-        const uint32_t dst = sS + copy_base + a * 8192 + ll.dst0;
+        const uint32_t dst = sS + a * 8192 + ll.dst0;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const bool tv = whole || tb + ll.lw + 8 * k < t1;
@@ -481,37 +474,43 @@ __global__ void __launch_bounds__(kThreads, 1) gr_kernel(const __grid_constant__
       }
       cp_async_commit();
       cp_async_wait(0);
-      publish(&full[rp.slot], lane);
-      rp.advance(kSets, S);
+      publish(&fullC[set], lane);
     }
     cp_async_wait(0);
   } else if (warp == kEpiWarps) {
     if (lane == 0) {
       const uint32_t idesc = make_idesc(128, NP, 1, 1);
-      RingPos rp;
-      rp.init(0, S);
+      RingPos rt;
+      rt.init(0, ST);
       bool ok = true;
       for (int s = 0; s < nst; ++s) {
-        if (!wait_bar(&full[rp.slot], rp.ph, &abort_s, L.err)) { ok = false; break; }
+        const int sc = s & (kSets - 1), pc = (s / kSets) & 1;
+        if (!wait_bar(&fullT[rt.slot], rt.ph, &abort_s, L.err) || !wait_bar(&fullC[sc], pc, &abort_s, L.err)) { ok = false; break; }
         fence_after_sync();
-        const uint32_t lAddr = smem_u32(sm + (size_t)rp.slot * stage_bytes), rAddr = lAddr + 2 * 8192;
-        const uint64_t ad = make_desc(lAddr, 8192, 1024), bd = make_desc(rAddr, 8192, 1024);
+        const uint32_t tAddr = smem_u32(ringT + (size_t)rt.slot * tbytes), cAddr = smem_u32(ringC + (size_t)sc * cbytes);
+        const uint32_t lAddr = L.tma_is_L ? tAddr : cAddr, rAddr = L.tma_is_L ? cAddr : tAddr;
+        const uint64_t bd = make_desc(rAddr, 8192, 1024);
+        for (int blk = 0; blk < MB; ++blk) {
+          const uint64_t ad = make_desc(lAddr + blk * 2 * 8192, 8192, 1024);
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) mma_bf16(tmem, ad + kk * 128, bd + kk * 128, idesc, (s | kk) != 0);
-        commit(&empty[rp.slot]);
-        rp.advance(1, S);
+          for (int kk = 0; kk < 4; ++kk) mma_bf16(tmem + blk * NP, ad + kk * 128, bd + kk * 128, idesc, (s | kk) != 0);
+        }
+        commit(&emptyT[rt.slot]);
+        commit(&emptyC[sc]);
+        rt.advance(1, ST);
       }
       if (ok) commit(&done);
     }
   } else {
     if (wait_bar_warp(&done, 0, &abort_s, L.err)) {
       fence_after_sync();
-      const int mi = mb * 128 + tid;                                  // index in the M space
-      const int m = L.tma_is_L ? (mi < L.M ? unpad_index(mi, L.Ap, L.dp, L.d, L.C) : -1) : (mi < L.M ? mi : -1);
       const int ones = L.tma_is_L ? L.pvalid : (L.d < L.dp ? L.d : -1);   // N index of the ones column
+      for (int blk = 0; blk < MB; ++blk)
       for (int c0 = 0; c0 < NP; c0 += 32) {
+        const int mi = (mb + blk) * 128 + tid;                          // index in the M space
+        const int m = L.tma_is_L ? (mi < L.M ? unpad_index(mi, L.Ap, L.dp, L.d, L.C) : -1) : (mi < L.M ? mi : -1);
         uint32_t v[32];
-        tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + c0, v);
+        tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + blk * NP + c0, v);
         tmem_ld_wait();
         if (m >= 0) {
           float* orow = L.out + (long long)m * L.C;
@@ -678,14 +677,18 @@ int launch_gt(const GTLaunch& L, int nsplits, cudaStream_t st, const char* name)
 
 int launch_gr(const GRLaunch& L, cudaStream_t st, const char* name) {
   GRLaunch Lc = L;
-  Lc.nstages = (int)((215 * 1024) / ((size_t)(2 + L.NP / 64) * 8192));
-  if (Lc.nstages > 6) Lc.nstages = 6;
-  if (Lc.nstages < 3) return GSWA_ERR_UNSUPPORTED;
-  const size_t smem = 1024 + (size_t)Lc.nstages * (2 + L.NP / 64) * 8192 + 64;
+  if (Lc.mbpc < 1 || Lc.mbpc * L.NP > 512) Lc.mbpc = 1;
+  const int latoms = 2 * Lc.mbpc, ratoms = L.NP / 64;
+  const size_t tbytes = (size_t)(L.tma_is_L ? latoms : ratoms) * 8192, cbytes = (size_t)(L.tma_is_L ? ratoms : latoms) * 8192;
+  const size_t budget = 215 * 1024;
+  if (budget < 1024 + kSets * cbytes + 2 * tbytes) return GSWA_ERR_UNSUPPORTED;
+  Lc.nstages = (int)((budget - 1024 - kSets * cbytes) / tbytes);      // TMA ring depth
+  if (Lc.nstages > 8) Lc.nstages = 8;
+  const size_t smem = 1024 + (size_t)Lc.nstages * tbytes + kSets * cbytes + 64;
   if (cudaFuncSetAttribute(gr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return check_launch();
-  const int mblocks = (L.M + 127) / 128;
-  { KernelScope ks_(name, st); gr_kernel<<<dim3(L.nsplit, mblocks), kThreads, smem, st>>>(Lc); }
+  const int mblocks = ((L.M + 127) / 128 + Lc.mbpc - 1) / Lc.mbpc;
+  { KernelScope ks_(name, st); gr_kernel<<<dim3(L.nsplit, mblocks), kThreadsR, smem, st>>>(Lc); }
   return check_launch();
 }
 

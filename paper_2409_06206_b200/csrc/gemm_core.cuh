@@ -11,7 +11,8 @@ using namespace umma;
 
 
 constexpr int kEpiWarps = 4, kLoadWarps = 8;
-constexpr int kThreads = 32 * (kEpiWarps + 1 + kLoadWarps);   // 416 (gr_kernel)
+constexpr int kThreads = 32 * (kEpiWarps + 1 + kLoadWarps);   // 416
+constexpr int kThreadsR = kThreads + 32;                      // gr_kernel: one more warp, the TMA producer
 // gw_kernel / gt_kernel drain TMEM with two warps per 32-lane quadrant (a warp may only read the
 // TMEM lanes 32*(warp%4) .. +31): warps 0-7 epilogue, warp 8 MMA issue, warps 9-16 loaders.
 constexpr int kEpi2 = 8;
@@ -81,7 +82,10 @@ __host__ __device__ inline uint32_t pow2_cols(int n) {
 // warps form four sets of two warps; set q fills ring steps q, q+4, q+8, ...: it waits until the
 // tensor core has released the slot, issues its asynchronous copies, waits for them to land, and
 // publishes the slot at once.  Four steps of loads are therefore in flight per SM and a slot becomes
-// visible to the MMA warp as soon as its own data has arrived.
+// visible to the MMA warp as soon as its own data has arrived.  The ring must have at least as many
+// slots as there are sets: then the set that refills a slot has already seen the release of the
+// slot's last-but-one use, so a parity wait can never be satisfied by a stale phase and two sets
+// never arrive on the same `full` barrier in one phase.
 constexpr int kSets = 4;                      // loader sets
 constexpr int kAtomBytes = 128 * 128;         // one ring slot
 
