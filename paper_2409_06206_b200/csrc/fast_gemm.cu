@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
   constexpr int kPiece = 32 * DP * 2;                      // 32 rows of one output block: contiguous in global memory
   unsigned char* stg = ring + (size_t)S * kAtomBytes;      // two pieces per epilogue warp
   float* sBias = reinterpret_cast<float*>(stg + (size_t)kEpi2 * 2 * kPiece);
-  __shared__ uint64_t full[8], empty[8], tfull, tempty[8];
+  __shared__ uint64_t full[8], empty[8], tfull[8], tempty[8];
   __shared__ uint32_t tmem_s;
   __shared__ int abort_s;
 
@@ -49,11 +49,15 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
   if (tid == 0) {
     abort_s = 0;
     for (int i = 0; i < 8; ++i) { mbar_init(&full[i], 2); mbar_init(&empty[i], 1); }
-    mbar_init(&tfull, 1);
-    for (int i = 0; i < 8; ++i) mbar_init(&tempty[i], kEpi2);
+    for (int i = 0; i < 8; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], kEpi2); }
     mbar_init_fence();
   }
-  const uint32_t tcols = pow2_cols(NT);
+  // TMEM holds a ring of RC accumulator chunks of cw columns; a tile takes nchunks consecutive ring
+  // positions, so the MMAs of the next tile start while this tile's chunks are still being drained.
+  // (With several chunks per tile the overlap only makes the MMAs and the epilogue fight for shared-memory
+  // bandwidth -- measured slower -- so the ring is then exactly one tile deep.)
+  const int RC = u.nchunks > 1 ? u.nchunks : (512 / u.cw < 8 ? 512 / u.cw : 8);
+  const uint32_t tcols = pow2_cols(RC * u.cw);
   if (warp == kEpi2) tmem_alloc(&tmem_s, tcols);
   fence_before_sync();
   __syncthreads();
@@ -129,12 +133,12 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
       const uint64_t a0 = make_desc(smem_u32(ring), 16, 1024), b0 = make_desc(smem_u32(sB), 16, 1024);
       RingPos rp;
       rp.init(0, S);
-      int it = 0;
+      int q = 0, qph = 0, qlast = 0;                               // ring position of the next chunk and its phase
       bool ok = true;
-      for (long long tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
+      for (long long tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         int slot_a[NA];
         for (int c = 0; c < u.nchunks && ok; ++c) {
-          if (!wait_bar(&tempty[c], (it & 1) ^ 1, &abort_s, L.err)) { ok = false; break; }
+          if (!wait_bar(&tempty[q], qph ^ 1, &abort_s, L.err)) { ok = false; break; }
           fence_after_sync();
 #pragma unroll
           for (int atom = 0; atom < NA; ++atom) {
@@ -147,13 +151,15 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
             const uint64_t ad = a0 + (uint64_t)((slot_a[atom] * kAtomBytes) >> 4);
             const uint64_t bd = b0 + (uint64_t)(((atom * NT + c * u.cw) * 128) >> 4);
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) mma_bf16(tmem + c * u.cw, ad + 2 * kk, bd + 2 * kk, idesc, (atom | kk) != 0);
+            for (int kk = 0; kk < 4; ++kk) mma_bf16(tmem + q * u.cw, ad + 2 * kk, bd + 2 * kk, idesc, (atom | kk) != 0);
           }
+          qlast = q;
+          if (++q == RC) { q = 0; qph ^= 1; }
         }
         if (!ok) break;
 #pragma unroll
         for (int atom = 0; atom < NA; ++atom) commit(&empty[slot_a[atom]]);
-        commit(&tfull);
+        commit(&tfull[qlast]);                     // one completion signal per tile, on its last chunk
       }
     }
   } else {
@@ -165,20 +171,25 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
     const int nblk = u.cw / DP;
     unsigned char* mystg = stg + (size_t)warp * 2 * kPiece;
     const uint32_t mystgA = smem_u32(mystg);
-    int it = 0, nst = 0;
+    int nst = 0, q = 0, qph = 0;                  // q, qph: ring position of the next chunk and its phase
     bool ok = true;
-    for (long long tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
+    for (long long tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
       const long long win = 2 * tile + (quad >> 1);
       const bool valid = win < u.n_windows;
       __nv_bfloat16* obase = u.out + win * u.win_stride + (quad & 1) * 32 * DP;
-      if (!wait_bar_warp(&tfull, it & 1, &abort_s, L.err)) break;
-      fence_after_sync();
+      {
+        // the tile is complete when its last chunk is (MMAs finish in issue order)
+        int ql = q + u.nchunks - 1, pl = qph;
+        if (ql >= RC) { ql -= RC; pl ^= 1; }
+        if (!wait_bar_warp(&tfull[ql], pl, &abort_s, L.err)) break;
+      }
       for (int c = 0; c < u.nchunks; ++c) {
+        fence_after_sync();
         for (int blk = 0; blk < nblk; ++blk) {
           const int gb = c * nblk + blk;
           if ((gb & 1) != half) continue;          // the two warps of a quadrant alternate blocks
           uint32_t v[DP];
-          const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + gb * DP;
+          const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + q * u.cw + blk * DP;
           if constexpr (DP == 32) tmem_ld32(taddr, v); else tmem_ld16(taddr, v);
           const int buf = nst & 1;
           if (nst >= 2) {                          // the copy that last read this buffer has finished reading
@@ -209,7 +220,8 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
         }
         fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&tempty[c]);
+        if (lane == 0) mbar_arrive(&tempty[q]);
+        if (++q == RC) { q = 0; qph ^= 1; }
       }
     }
     if (lane == 0) bulk_wait_all();
