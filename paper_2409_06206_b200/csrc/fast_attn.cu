@@ -48,22 +48,22 @@ __global__ void __launch_bounds__(384, 2) attn_fwd_kernel(const __grid_constant_
   if (win < g.n_windows) load_tiles<DP>(sm, L.qkv + u.qkv_off + win * u.qkv_wstride, nh_u * 3, tid, nt);
   cp_async_commit();
   for (int buf = 0; win < g.n_windows; win += gridDim.x, buf ^= 1) {
+    int* tok = tok2 + buf * 64;
+    unsigned char* reg = reg2 + buf * 64;
+    const WinCtx wc = window_setup(g, u.s, win, tok, reg, tid);
+    cp_async_wait_all();
+    __syncthreads();   // this window's tiles and maps are complete; every warp has left the previous window,
+                       // so the other buffer may be refilled
     const long long nxt = win + gridDim.x;
     if (nxt < g.n_windows)
       load_tiles<DP>(sm + (size_t)(buf ^ 1) * tile_bytes, L.qkv + u.qkv_off + nxt * u.qkv_wstride, nh_u * 3, tid, nt);
     cp_async_commit();
-    int* tok = tok2 + buf * 64;
-    unsigned char* reg = reg2 + buf * 64;
-    const WinCtx wc = window_setup(g, u.s, win, tok, reg, tid);
-    cp_async_wait_1();
-    __syncthreads();
 
     unsigned char* tiles = sm + (size_t)buf * tile_bytes;
     const uint32_t q_base = smem_u32(tiles + (size_t)(hl * 3 + 0) * 64 * DP * 2);
     fwd_window<DP>(q_base, q_base + 64 * DP * 2, q_base + 2 * 64 * DP * 2, tab + hl * 225, tok, reg, wc.masked, r0, lane,
                    ostg, L.A, g.nh * DP, h, g.d,
                    L.Lt != nullptr ? L.Lt + u.l_off + win * u.l_wstride + hl * 64 : nullptr);
-    __syncthreads();   // every warp is done with this buffer before the next iteration refills it
   }
   cp_async_wait_all();
 }
@@ -120,15 +120,16 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
   if (win < g.n_windows) fetch(win, 0);
   cp_async_commit();
   for (int buf = 0; win < g.n_windows; win += gridDim.x, buf ^= 1) {
-    const long long nxt = win + gridDim.x;
-    if (nxt < g.n_windows) fetch(nxt, buf ^ 1);
-    cp_async_commit();
     int* tok = tok2 + buf * 64;
     unsigned char* reg = reg2 + buf * 64;
     const float* Lrow = Lrow2 + buf * nh_u * 64;
     const WinCtx wc = window_setup(g, u.s, win, tok, reg, tid);
-    cp_async_wait_1();
-    __syncthreads();
+    cp_async_wait_all();
+    __syncthreads();   // this window's inputs are complete; every warp has left the previous window, so the
+                       // other input buffer, P and dS may be overwritten
+    const long long nxt = win + gridDim.x;
+    if (nxt < g.n_windows) fetch(nxt, buf ^ 1);
+    cp_async_commit();
     unsigned char* tiles = sm + (size_t)buf * in_bytes;
     const uint32_t q_base = smem_u32(tiles + (size_t)(hl * 3) * kTile);
     const uint32_t k_base = q_base + kTile, v_base = k_base + kTile;
@@ -222,7 +223,6 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
     // q was stored scaled by log2(e) (the scores live in the log2 domain): dK = dS^T q takes it back out
     store_tile<DP>(ostg, dk, kLn2, drow0 + Ap * 2, drow1 + Ap * 2, lane, -1);
     store_tile<DP>(ostg, dv, 1.f, drow0 + Ap * 4, drow1 + Ap * 4, lane, -1);
-    __syncthreads();   // tiles, P and dS of this window are no longer read
   }
   cp_async_wait_all();
 
