@@ -170,6 +170,25 @@ def test_stacked_inference_layers():
         x = round_to_bf16(x)
 
 
+def test_stacked_inference_full_size_image():
+    """The 512 x 512 inference image at full size: six layers with alternating group assignment run back to
+    back in inference mode; the first and the last layer are checked against the checker on the full image."""
+    import torch
+    from paper_2409_06206_b200.inputs import round_to_bf16
+    cfg = CONFIGS["c5"]
+    x = make_inputs(cfg, tensors=("x",))["x"]
+    for layer in range(cfg.layers):
+        inp = make_inputs(cfg, layer=layer, tensors=("w_qkv", "b_qkv", "w_proj", "b_proj", "bias_table"))
+        inp["x"] = x
+        got = run_gpu(cfg, inp, backward=False, layer=layer, inference=True)
+        assert np.isfinite(got["y"]).all()
+        if layer in (0, cfg.layers - 1):
+            ref = run_oracle(cfg, inp, backward=False, layer=layer)
+            assert rel_err(got["y"], ref["y"]) <= 2e-2
+        x = round_to_bf16(round_to_bf16(got["y"].astype(np.float32)) * np.float32(4.0))
+    torch.cuda.synchronize()
+
+
 def test_step_host_matches_device_path():
     import torch
     cfg = SWEEP[7]
