@@ -298,22 +298,6 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
   int rc = launch_prep(jobs, nj, st);
   if (rc) return rc;
 
-  // dO tiles = dy W^P restricted to each unit's heads, rows gathered in that group's window order
-  GWLaunch gw{};
-  gw.err = err;
-  for (int i = 0; i < nu; ++i) {
-    const Unit& u = units[i];
-    GWUnit& w = gw.u[i];
-    w.A = (const bf*)dy; w.lda = p.C; w.kvalid = p.C;
-    w.H = p.H; w.W = p.W; w.s = p.gs[u.g]; w.nW = p.nW; w.nWw = p.nWw; w.n_windows = geo.n_windows;
-    w.Bimg = (const unsigned char*)sc + bs.img[i];
-    w.bias = nullptr;
-    w.out = dO + geo.do_off[u.g] + (long long)(u.h0 - p.gh0[u.g]) * 64 * p.dp;
-    w.win_stride = (long long)p.gh[u.g] * 64 * p.dp;
-    w.nchunks = 1; w.cw = u.nheads * p.dp; w.q_every3 = 0; w.qscale = 1.f;
-  }
-  if ((rc = launch_gw(gw, nu, p.Cp, p.dp, st, "dattn_gemm"))) return rc;
-
   const int sms = 148;
   if (dw_proj || db_proj) {
     // dW^P = dy^T A (A fetched by TMA); db^P rides on the ones column of A when the head dim is padded
@@ -331,6 +315,23 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
     if ((rc = launch_gr(gr, st, "dwproj_gemm"))) return rc;
     if (db_proj && p.d == p.dp && (rc = launch_colsum_bf16((const bf*)dy, p.T, p.C, p.C, db_proj, st))) return rc;
   }
+
+  // (dW^P runs first so that the dO tiles written next are still in L2 when the attention kernel reads them)
+  // dO tiles = dy W^P restricted to each unit's heads, rows gathered in that group's window order
+  GWLaunch gw{};
+  gw.err = err;
+  for (int i = 0; i < nu; ++i) {
+    const Unit& u = units[i];
+    GWUnit& w = gw.u[i];
+    w.A = (const bf*)dy; w.lda = p.C; w.kvalid = p.C;
+    w.H = p.H; w.W = p.W; w.s = p.gs[u.g]; w.nW = p.nW; w.nWw = p.nWw; w.n_windows = geo.n_windows;
+    w.Bimg = (const unsigned char*)sc + bs.img[i];
+    w.bias = nullptr;
+    w.out = dO + geo.do_off[u.g] + (long long)(u.h0 - p.gh0[u.g]) * 64 * p.dp;
+    w.win_stride = (long long)p.gh[u.g] * 64 * p.dp;
+    w.nchunks = 1; w.cw = u.nheads * p.dp; w.q_every3 = 0; w.qscale = 1.f;
+  }
+  if ((rc = launch_gw(gw, nu, p.Cp, p.dp, st, "dattn_gemm"))) return rc;
 
   AttnLaunch al{};
   attn_units(p, geo, units, nu, &al);

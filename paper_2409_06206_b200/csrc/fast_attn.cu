@@ -44,18 +44,20 @@ __global__ void __launch_bounds__(384, 2) attn_fwd_kernel(const __grid_constant_
   const int p0 = r0 + gq;
   const int h = u.h0 + hl;
 
-  long long win = blockIdx.x;
-  if (win < g.n_windows) load_tiles<DP>(sm, L.qkv + u.qkv_off + win * u.qkv_wstride, nh_u * 3, tid, nt);
+  // Windows are visited from the last to the first: the kernel that produced the tiles wrote the last
+  // windows last, so they are the ones still resident in L2.
+  long long win = g.n_windows - 1 - blockIdx.x;
+  if (win >= 0) load_tiles<DP>(sm, L.qkv + u.qkv_off + win * u.qkv_wstride, nh_u * 3, tid, nt);
   cp_async_commit();
-  for (int buf = 0; win < g.n_windows; win += gridDim.x, buf ^= 1) {
+  for (int buf = 0; win >= 0; win -= gridDim.x, buf ^= 1) {
     int* tok = tok2 + buf * 64;
     unsigned char* reg = reg2 + buf * 64;
     const WinCtx wc = window_setup(g, u.s, win, tok, reg, tid);
     cp_async_wait_all();
     __syncthreads();   // this window's tiles and maps are complete; every warp has left the previous window,
                        // so the other buffer may be refilled
-    const long long nxt = win + gridDim.x;
-    if (nxt < g.n_windows)
+    const long long nxt = win - gridDim.x;
+    if (nxt >= 0)
       load_tiles<DP>(sm + (size_t)(buf ^ 1) * tile_bytes, L.qkv + u.qkv_off + nxt * u.qkv_wstride, nh_u * 3, tid, nt);
     cp_async_commit();
 
@@ -116,10 +118,11 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
     for (int e = tid; e < nh_u * 16; e += nt) cp_async16(smem_u32(ldst + 4 * e), lsrc + 4 * e);
   };
 
-  long long win = blockIdx.x;
-  if (win < g.n_windows) fetch(win, 0);
+  // last window first: the dO tiles written last by the preceding GEMM are still in L2
+  long long win = g.n_windows - 1 - blockIdx.x;
+  if (win >= 0) fetch(win, 0);
   cp_async_commit();
-  for (int buf = 0; win < g.n_windows; win += gridDim.x, buf ^= 1) {
+  for (int buf = 0; win >= 0; win -= gridDim.x, buf ^= 1) {
     int* tok = tok2 + buf * 64;
     unsigned char* reg = reg2 + buf * 64;
     const float* Lrow = Lrow2 + buf * nh_u * 64;
@@ -127,8 +130,8 @@ __global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant_
     cp_async_wait_all();
     __syncthreads();   // this window's inputs are complete; every warp has left the previous window, so the
                        // other input buffer, P and dS may be overwritten
-    const long long nxt = win + gridDim.x;
-    if (nxt < g.n_windows) fetch(nxt, buf ^ 1);
+    const long long nxt = win - gridDim.x;
+    if (nxt >= 0) fetch(nxt, buf ^ 1);
     cp_async_commit();
     unsigned char* tiles = sm + (size_t)buf * in_bytes;
     const uint32_t q_base = smem_u32(tiles + (size_t)(hl * 3) * kTile);
