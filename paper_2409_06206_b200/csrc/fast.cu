@@ -158,8 +158,17 @@ void fast_plan_sizes(Plan* p) {
   p->bwd_scratch = bwd_layout(*p, units, nu, tx).total;
 }
 
+// Work units of the attention kernels: one head per CTA when the unit table has room for every head (more,
+// smaller CTAs per SM hide each other's latency), otherwise the head ranges of the GEMM units.
 static void attn_units(const Plan& p, const FastGeom& geo, const Unit* units, int nu, AttnLaunch* L) {
   L->geo = geo;
+  Unit heads[kMaxUnits];
+  if (p.nh <= kMaxUnits) {
+    nu = 0;
+    for (int g = 0; g < p.G; ++g)
+      for (int h = 0; h < p.gh[g]; ++h) heads[nu++] = Unit{g, p.gh0[g] + h, 1};
+    units = heads;
+  }
   L->nunits = nu;
   for (int i = 0; i < nu; ++i) {
     const Unit& u = units[i];

@@ -22,8 +22,10 @@ namespace {
 // warp.  The q,k,v tiles of the next window are copied into the second buffer while the current
 // window is being computed.
 // ------------------------------------------------------------------------------------------
-template <int DP>
-__global__ void __launch_bounds__(384, 2) attn_fwd_kernel(const __grid_constant__ AttnLaunch L) {
+// HPU = heads per CTA the kernel is compiled for (1: one head per CTA, 128 threads, many CTAs per SM;
+// 3: up to three heads per CTA).
+template <int DP, int HPU>
+__global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 7 : 2) attn_fwd_kernel(const __grid_constant__ AttnLaunch L) {
   const AttnUnit& u = L.u[blockIdx.y];
   const FastGeom& g = L.geo;
   extern __shared__ __align__(128) unsigned char sm[];
@@ -73,8 +75,8 @@ __global__ void __launch_bounds__(384, 2) attn_fwd_kernel(const __grid_constant_
 // ------------------------------------------------------------------------------------------
 // backward: persistent CTAs stride over the windows of a unit
 // ------------------------------------------------------------------------------------------
-template <int DP>
-__global__ void __launch_bounds__(384, 1) attn_bwd_kernel(const __grid_constant__ AttnLaunch L) {
+template <int DP, int HPU>
+__global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 4 : 1) attn_bwd_kernel(const __grid_constant__ AttnLaunch L) {
   const AttnUnit& u = L.u[blockIdx.y];
   const FastGeom& g = L.geo;
   extern __shared__ __align__(128) unsigned char sm[];
@@ -254,51 +256,68 @@ size_t bwd_smem(int nheads) {
          (size_t)nheads * 4 * 16 * DP * 2;
 }
 
-template <int DP>
-int launch_fwd_t(const AttnLaunch& L, cudaStream_t st) {
-  int maxh = 0;
-  for (int i = 0; i < L.nunits; ++i) maxh = L.u[i].nheads > maxh ? L.u[i].nheads : maxh;
+// CTAs per SM the hardware will co-schedule for this kernel and launch shape.
+template <typename K>
+int blocks_per_sm(K kernel, int threads, size_t smem) {
+  int n = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, smem) != cudaSuccess || n < 1) {
+    (void)cudaGetLastError();
+    n = 1;
+  }
+  return n;
+}
+
+template <int DP, int HPU>
+int launch_fwd_t(const AttnLaunch& L, int maxh, cudaStream_t st) {
   const size_t smem = fwd_smem<DP>(maxh);
-  if (cudaFuncSetAttribute(attn_fwd_kernel<DP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+  if (cudaFuncSetAttribute(attn_fwd_kernel<DP, HPU>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return check_launch();
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int per_sm = smem * 2 <= 220 * 1024 ? 2 : 1;
+  const int per_sm = blocks_per_sm(attn_fwd_kernel<DP, HPU>, maxh * 128, smem);
   long long gx = (long long)sms * per_sm / L.nunits;
   if (gx < 1) gx = 1;
   if (gx > L.geo.n_windows) gx = L.geo.n_windows;
   { KernelScope ks_("attn_fwd", st);
-    attn_fwd_kernel<DP><<<dim3((unsigned)gx, L.nunits), maxh * 128, smem, st>>>(L); }
+    attn_fwd_kernel<DP, HPU><<<dim3((unsigned)gx, L.nunits), maxh * 128, smem, st>>>(L); }
   return check_launch();
 }
 
-template <int DP>
-int launch_bwd_t(const AttnLaunch& L, cudaStream_t st) {
-  int maxh = 0;
-  for (int i = 0; i < L.nunits; ++i) maxh = L.u[i].nheads > maxh ? L.u[i].nheads : maxh;
+template <int DP, int HPU>
+int launch_bwd_t(const AttnLaunch& L, int maxh, cudaStream_t st) {
   const size_t smem = bwd_smem<DP>(maxh);
-  if (cudaFuncSetAttribute(attn_bwd_kernel<DP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+  if (cudaFuncSetAttribute(attn_bwd_kernel<DP, HPU>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return check_launch();
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int per_sm = smem * 2 <= 220 * 1024 ? 2 : 1;
+  const int per_sm = blocks_per_sm(attn_bwd_kernel<DP, HPU>, maxh * 128, smem);
   long long gx = (long long)sms * per_sm / L.nunits;
   if (gx < 1) gx = 1;
   if (gx > L.geo.n_windows) gx = L.geo.n_windows;
   { KernelScope ks_("attn_bwd", st);
-    attn_bwd_kernel<DP><<<dim3((unsigned)gx, L.nunits), maxh * 128, smem, st>>>(L); }
+    attn_bwd_kernel<DP, HPU><<<dim3((unsigned)gx, L.nunits), maxh * 128, smem, st>>>(L); }
   return check_launch();
+}
+
+int max_heads(const AttnLaunch& L) {
+  int maxh = 0;
+  for (int i = 0; i < L.nunits; ++i) maxh = L.u[i].nheads > maxh ? L.u[i].nheads : maxh;
+  return maxh;
 }
 
 }  // namespace
 
 int launch_attn_fwd(const AttnLaunch& L, cudaStream_t st) {
-  return L.geo.dp == 32 ? launch_fwd_t<32>(L, st) : launch_fwd_t<16>(L, st);
+  const int maxh = max_heads(L);
+  if (maxh == 1) return L.geo.dp == 32 ? launch_fwd_t<32, 1>(L, 1, st) : launch_fwd_t<16, 1>(L, 1, st);
+  return L.geo.dp == 32 ? launch_fwd_t<32, 3>(L, maxh, st) : launch_fwd_t<16, 3>(L, maxh, st);
 }
 int launch_attn_bwd(const AttnLaunch& L, cudaStream_t st) {
-  return L.geo.dp == 32 ? launch_bwd_t<32>(L, st) : launch_bwd_t<16>(L, st);
+  const int maxh = max_heads(L);
+  if (maxh == 1) return L.geo.dp == 32 ? launch_bwd_t<32, 1>(L, 1, st) : launch_bwd_t<16, 1>(L, 1, st);
+  return L.geo.dp == 32 ? launch_bwd_t<32, 3>(L, maxh, st) : launch_bwd_t<16, 3>(L, maxh, st);
 }
 
 }  // namespace gswa
