@@ -67,3 +67,15 @@ def test_argument_errors_are_reported_before_any_launch():
     assert gb.gswa_launch_count() == n0
     assert gb.gswa_step_host_arena_bytes(d) > 0
     assert "NULL" in gb.gswa_status_string(-1) and gb.gswa_status_string(0) == "ok"
+
+
+def test_binding_constants_match_the_header():
+    text = open(os.path.join(ROOT, "include", "gswa.h")).read()
+    vals = dict(re.findall(r"(GSWA_[A-Z0-9_]+)\s*=\s*(-?\d+)u?", text))
+    assert int(vals["GSWA_FLAG_ACCUMULATE"]) == gb.FLAG_ACCUMULATE
+    assert int(vals["GSWA_FLAG_GENERIC"]) == gb.FLAG_GENERIC
+    assert int(vals["GSWA_FLAG_FUSED_FWD"]) == gb.FLAG_FUSED_FWD
+    assert int(vals["GSWA_F32"]) == gb.GSWA_F32 and int(vals["GSWA_BF16"]) == gb.GSWA_BF16
+    m = re.search(r"GSWA_STATIC_SCRATCH_BYTES \((\d+)u << (\d+)\)", text)
+    assert int(m.group(1)) << int(m.group(2)) == gb.STATIC_SCRATCH_BYTES
+    assert set(gb.EXPORTS) == set(_declared())
