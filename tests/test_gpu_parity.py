@@ -80,6 +80,39 @@ def test_small_shapes_forward_backward(cfg):
     assert_close(got, ref, cfg.dtype)
 
 
+def _random_fast_path_shapes(n, seed=1234):
+    """Seeded random layer shapes that the tensor-core path accepts (window 8, even head dim <= 32, padded
+    attention width >= 64): odd window counts, every shift, one to four groups, all K paddings."""
+    rng = np.random.default_rng(seed)
+    out = []
+    choices = [(64, 2), (64, 4), (96, 3), (96, 6), (120, 4), (128, 4), (128, 8), (144, 6), (180, 6), (192, 6), (224, 7),
+               (240, 8), (252, 7), (56, 4), (72, 6)]
+    while len(out) < n:
+        C, nh = choices[int(rng.integers(len(choices)))]
+        d = C // nh
+        if d % 2 or d > 32 or nh * (16 if d <= 16 else 32) < 64:
+            continue
+        G = int(rng.integers(1, min(4, nh) + 1))
+        cuts = sorted(rng.choice(np.arange(1, nh), size=G - 1, replace=False).tolist()) if G > 1 else []
+        gh = tuple(int(b - a) for a, b in zip([0] + cuts, cuts + [nh]))
+        gs = tuple(int(rng.integers(0, 8)) for _ in range(G))
+        B, H, W = int(rng.integers(1, 4)), 8 * int(rng.integers(1, 5)), 8 * int(rng.integers(1, 6))
+        out.append(_mk("r%d" % len(out), B, H, W, C, nh, 8, gh, gs, "bf16", seed=100 + len(out)))
+    return out
+
+
+RANDOM_SHAPES = _random_fast_path_shapes(14)
+
+
+@pytest.mark.parametrize("cfg", RANDOM_SHAPES, ids=["%s-B%dx%dx%d-C%d-h%s-s%s" % (c.name, c.B, c.H, c.W, c.C, "".join(map(str, c.group_heads)),
+                                                   "".join(map(str, c.group_shift))) for c in RANDOM_SHAPES])
+def test_random_shapes_tensor_core_path(cfg):
+    inp = make_inputs(cfg)
+    ref = run_oracle(cfg, inp)
+    assert_close(run_gpu(cfg, inp), ref, cfg.dtype)
+    assert_close(run_gpu(cfg, inp, flags=gb.FLAG_FUSED_FWD), ref, cfg.dtype)
+
+
 @pytest.mark.parametrize("cfg", [SWEEP[2], SWEEP[7], SWEEP[8]], ids=["f32", "bf16-c60", "bf16-c180"])
 def test_generic_kernels_forced(cfg):
     inp = make_inputs(cfg)
