@@ -258,7 +258,7 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
 
     AttnLaunch al{};
     attn_units(p, geo, units, nu, &al);
-    al.qkv = qkv; al.table = (const bf*)table; al.A = A; al.Lt = want_L ? Lt : nullptr;
+    al.qkv = qkv; al.table = (const bf*)table; al.A = A; al.Lt = want_L ? Lt : nullptr; al.err = err;
     al.scale = 1.0f / sqrtf((float)p.d);
     if ((rc = launch_attn_fwd(al, st))) return rc;
   }
@@ -345,7 +345,7 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
   AttnLaunch al{};
   attn_units(p, geo, units, nu, &al);
   al.qkv = qkv; al.table = (const bf*)table; al.Lt = const_cast<float*>(Lt); al.dO = dO; al.dqkv = dqkv;
-  al.dtable = dtable; al.scale = 1.0f / sqrtf((float)p.d);
+  al.dtable = dtable; al.scale = 1.0f / sqrtf((float)p.d); al.err = err;
   if ((rc = launch_attn_bwd(al, st))) return rc;
 
   if (dx) {

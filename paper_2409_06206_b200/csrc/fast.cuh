@@ -172,6 +172,7 @@ struct AttnLaunch {
   const __nv_bfloat16* dO;     // bwd: dO tiles
   __nv_bfloat16* dqkv;         // bwd: [T, 3*Ap] out
   float* dtable;               // bwd: [(2M-1)^2, nh] float, atomics; or nullptr
+  int* err;                    // device error word (set when a bounded wait gives up)
   float scale;
 };
 int launch_attn_fwd(const AttnLaunch& L, cudaStream_t st);

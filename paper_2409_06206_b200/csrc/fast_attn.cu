@@ -38,30 +38,42 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 7 : 2) attn_fwd_kernel(c
   unsigned char* ostg = sm + 2 * (size_t)tile_bytes + (((size_t)nh_u * 225 * 4 + 128 * 4 + 128 + 15) & ~(size_t)15) +
                         (size_t)warp * 16 * DP * 2;                 // this warp's 16 x DP output staging block
   const int nt = nh_u * 128;
+  __shared__ uint64_t ldbar[2];
+  if (tid == 0) {
+    umma::mbar_init(&ldbar[0], 1);
+    umma::mbar_init(&ldbar[1], 1);
+    umma::mbar_init_fence();
+  }
+  __syncthreads();
   if (tid >= nt) return;
 
   for (int e = tid; e < nh_u * 225; e += nt)
     tab[e] = __bfloat162float(L.table[(e % 225) * g.nh + u.h0 + e / 225]) * kLog2e;
-  const int hl = warp >> 2, r0 = (warp & 3) * 16, gq = lane >> 2, t = lane & 3;
-  const int p0 = r0 + gq;
+  const int hl = warp >> 2, r0 = (warp & 3) * 16;
   const int h = u.h0 + hl;
 
   // Windows are visited from the last to the first: the kernel that produced the tiles wrote the last
   // windows last, so they are the ones still resident in L2.
+  // One window's q,k,v tile images are contiguous in global memory and already laid out as the kernel
+  // wants them: one bulk asynchronous copy per window, counted in bytes on a barrier per buffer.
+  auto fetch = [&](long long w, int b) {
+    if (tid == 0) {
+      umma::fence_proxy_async();
+      umma::mbar_arrive_expect_tx(&ldbar[b], (uint32_t)tile_bytes);
+      umma::bulk_load(smem_u32(sm + (size_t)b * tile_bytes), L.qkv + u.qkv_off + w * u.qkv_wstride, (uint32_t)tile_bytes, &ldbar[b]);
+    }
+  };
   long long win = g.n_windows - 1 - blockIdx.x;
-  if (win >= 0) load_tiles<DP>(sm, L.qkv + u.qkv_off + win * u.qkv_wstride, nh_u * 3, tid, nt);
-  cp_async_commit();
-  for (int buf = 0; win >= 0; win -= gridDim.x, buf ^= 1) {
+  if (win >= 0) fetch(win, 0);
+  for (int buf = 0, it = 0; win >= 0; win -= gridDim.x, buf ^= 1, ++it) {
     int* tok = tok2 + buf * 64;
     unsigned char* reg = reg2 + buf * 64;
     const WinCtx wc = window_setup(g, u.s, win, tok, reg, tid);
-    cp_async_wait_all();
+    if (!umma::mbar_wait(&ldbar[buf], (it >> 1) & 1) && L.err != nullptr) atomicExch(L.err, 1);
     __syncthreads();   // this window's tiles and maps are complete; every warp has left the previous window,
                        // so the other buffer may be refilled
     const long long nxt = win - gridDim.x;
-    if (nxt >= 0)
-      load_tiles<DP>(sm + (size_t)(buf ^ 1) * tile_bytes, L.qkv + u.qkv_off + nxt * u.qkv_wstride, nh_u * 3, tid, nt);
-    cp_async_commit();
+    if (nxt >= 0) fetch(nxt, buf ^ 1);
 
     unsigned char* tiles = sm + (size_t)buf * tile_bytes;
     const uint32_t q_base = smem_u32(tiles + (size_t)(hl * 3 + 0) * 64 * DP * 2);
@@ -69,7 +81,6 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 7 : 2) attn_fwd_kernel(c
                    ostg, L.A, g.nh * DP, h, g.d,
                    L.Lt != nullptr ? L.Lt + u.l_off + win * u.l_wstride + hl * 64 : nullptr);
   }
-  cp_async_wait_all();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -94,6 +105,13 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 4 : 1) attn_bwd_kernel(c
   unsigned char* ostg = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(reg2 + 128) + 15) & ~(uintptr_t)15) +
                         (size_t)warp * 16 * DP * 2;              // this warp's 16 x DP output staging block
   const int nt = nh_u * 128;
+  __shared__ uint64_t ldbar[2];
+  if (tid == 0) {
+    umma::mbar_init(&ldbar[0], 1);
+    umma::mbar_init(&ldbar[1], 1);
+    umma::mbar_init_fence();
+  }
+  __syncthreads();
   if (tid >= nt) return;
 
   for (int e = tid; e < nh_u * 225; e += nt) {
@@ -110,31 +128,33 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 4 : 1) attn_bwd_kernel(c
 #pragma unroll
   for (int j = 0; j < 8; ++j) dsum[j][0] = dsum[j][1] = dsum[j][2] = dsum[j][3] = 0.f;
 
-  // copies of one window's inputs into buffer `b` (asynchronous)
+  // One window's inputs (q,k,v tile images, dO tile images, row log-sum-exp) are three contiguous runs in
+  // global memory: three bulk asynchronous copies per window, counted in bytes on a barrier per buffer.
   auto fetch = [&](long long w, int b) {
-    unsigned char* dst = sm + (size_t)b * in_bytes;
-    load_tiles<DP>(dst, L.qkv + u.qkv_off + w * u.qkv_wstride, nh_u * 3, tid, nt);
-    load_tiles<DP>(dst + (size_t)nh_u * 3 * kTile, L.dO + u.do_off + w * u.do_wstride, nh_u, tid, nt);
-    const float* lsrc = L.Lt + u.l_off + w * u.l_wstride;
-    float* ldst = Lrow2 + b * nh_u * 64;
-    for (int e = tid; e < nh_u * 16; e += nt) cp_async16(smem_u32(ldst + 4 * e), lsrc + 4 * e);
+    if (tid == 0) {
+      const uint32_t qb = (uint32_t)nh_u * 3 * kTile, ob = (uint32_t)nh_u * kTile, lb = (uint32_t)nh_u * 64 * 4;
+      unsigned char* dst = sm + (size_t)b * in_bytes;
+      umma::fence_proxy_async();
+      umma::mbar_arrive_expect_tx(&ldbar[b], qb + ob + lb);
+      umma::bulk_load(smem_u32(dst), L.qkv + u.qkv_off + w * u.qkv_wstride, qb, &ldbar[b]);
+      umma::bulk_load(smem_u32(dst + qb), L.dO + u.do_off + w * u.do_wstride, ob, &ldbar[b]);
+      umma::bulk_load(smem_u32(Lrow2 + b * nh_u * 64), L.Lt + u.l_off + w * u.l_wstride, lb, &ldbar[b]);
+    }
   };
 
   // last window first: the dO tiles written last by the preceding GEMM are still in L2
   long long win = g.n_windows - 1 - blockIdx.x;
   if (win >= 0) fetch(win, 0);
-  cp_async_commit();
-  for (int buf = 0; win >= 0; win -= gridDim.x, buf ^= 1) {
+  for (int buf = 0, it = 0; win >= 0; win -= gridDim.x, buf ^= 1, ++it) {
     int* tok = tok2 + buf * 64;
     unsigned char* reg = reg2 + buf * 64;
     const float* Lrow = Lrow2 + buf * nh_u * 64;
     const WinCtx wc = window_setup(g, u.s, win, tok, reg, tid);
-    cp_async_wait_all();
+    if (!umma::mbar_wait(&ldbar[buf], (it >> 1) & 1) && L.err != nullptr) atomicExch(L.err, 1);
     __syncthreads();   // this window's inputs are complete; every warp has left the previous window, so the
                        // other input buffer, P and dS may be overwritten
     const long long nxt = win - gridDim.x;
     if (nxt >= 0) fetch(nxt, buf ^ 1);
-    cp_async_commit();
     unsigned char* tiles = sm + (size_t)buf * in_bytes;
     const uint32_t q_base = smem_u32(tiles + (size_t)(hl * 3) * kTile);
     const uint32_t k_base = q_base + kTile, v_base = k_base + kTile;
@@ -229,7 +249,6 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 4 : 1) attn_bwd_kernel(c
     store_tile<DP>(ostg, dk, kLn2, drow0 + Ap * 2, drow1 + Ap * 2, lane, -1);
     store_tile<DP>(ostg, dv, 1.f, drow0 + Ap * 4, drow1 + Ap * 4, lane, -1);
   }
-  cp_async_wait_all();
 
   // ---- gradient of the bias table: fold this CTA's summed dS through the relative-position map
   if (L.dtable != nullptr) {

@@ -161,5 +161,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const void* tmap,
       : "memory");
 }
 
+// Bulk asynchronous copy global -> shared (sizes and addresses multiples of 16 bytes); completion is counted in
+// bytes on `bar` (the issuing thread first arrives with mbar_arrive_expect_tx).  No multicast.
+__device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_dst),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
 }  // namespace umma
 }  // namespace gswa
