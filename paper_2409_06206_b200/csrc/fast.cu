@@ -346,7 +346,24 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
   attn_units(p, geo, units, nu, &al);
   al.qkv = qkv; al.table = (const bf*)table; al.Lt = const_cast<float*>(Lt); al.dO = dO; al.dqkv = dqkv;
   al.dtable = dtable; al.scale = 1.0f / sqrtf((float)p.d); al.err = err;
-  if ((rc = launch_attn_bwd(al, st))) return rc;
+  bool one_head_units = true;
+  for (int i = 0; i < al.nunits; ++i) one_head_units = one_head_units && al.u[i].nheads == 1;
+  if (one_head_units && !(p.flags & GSWA_FLAG_WARP_MMA_ATTN)) {
+    if ((rc = make_tmap_window(&al.tm_out, dqkv, (long long)p.B * p.H, p.W, 3 * p.Ap, p.dp, 8, 8, true))) return rc;
+    // A window of a shifted group that wraps around the image edge is stored as four boxes.  Their shared-
+    // memory sources must start on 128-byte boundaries, which an even shift guarantees; units with another
+    // shift store such windows row by row.
+    al.wrap_s = 0;
+    for (int i = 0; i < al.nunits && al.wrap_s == 0; ++i)
+      if (al.u[i].s > 0 && al.u[i].s % 2 == 0) al.wrap_s = al.u[i].s;
+    if (al.wrap_s > 0) {
+      const int e = 8 - al.wrap_s, s = al.wrap_s;
+      for (int k = 0; k < 4; ++k)
+        if ((rc = make_tmap_window(&al.tm_wrap[k], dqkv, (long long)p.B * p.H, p.W, 3 * p.Ap, p.dp, (k & 1) ? s : e, (k & 2) ? s : e, false)))
+          return rc;
+    }
+    if ((rc = launch_attn_bwd_tc(al, st))) return rc;
+  } else if ((rc = launch_attn_bwd(al, st))) return rc;
 
   if (dx) {
     GTLaunch gt{};

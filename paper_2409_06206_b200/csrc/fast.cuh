@@ -139,6 +139,11 @@ int launch_gt(const GTLaunch& L, int nsplits, cudaStream_t st, const char* name)
 int launch_gr(const GRLaunch& L, cudaStream_t st, const char* name);
 // Tensor map of a padded token-major bf16 buffer [rows, cols]: box 64 columns x box_rows rows, 128-byte swizzle.
 int make_tmap(CUtensorMap* tm, const void* base, long long rows, int cols, int box_rows);
+// Tensor map of a padded token-major bf16 buffer [B*H image rows, W, cols] for stores of a block of
+// box_h x box_w tokens x dp columns.  Shared-memory side: rows of dp elements in box order, either with
+// the tile_off swizzle (8 x 8 boxes: the [64][dp] tile image) or unswizzled.
+int make_tmap_window(CUtensorMap* tm, const void* base, long long img_rows, int W, int cols, int dp, int box_w, int box_h,
+                     bool swizzled);
 
 // Weight images (shared-memory images of the B operands, built once per call by a small kernel).
 enum PrepMode { PREP_QKV = 0, PREP_PROJ_T = 1, PREP_PROJ = 2, PREP_QKV_T = 3 };
@@ -162,6 +167,10 @@ struct AttnUnit {
   long long qkv_wstride, do_wstride, l_wstride;
 };
 struct AttnLaunch {
+  CUtensorMap tm_out;          // window-block stores into dqkv (tcgen05 backward only)
+  CUtensorMap tm_wrap[4];      // the four pieces of a window that wraps around the image edge (shift wrap_s):
+                               // [2 * (lower rows) + (right columns)], boxes of (8-s | s) x (8-s | s) tokens
+  int wrap_s;                  // shift the pieces were cut for (an even shift of some unit), or 0
   FastGeom geo;
   AttnUnit u[kMaxUnits];
   int nunits;
@@ -177,6 +186,8 @@ struct AttnLaunch {
 };
 int launch_attn_fwd(const AttnLaunch& L, cudaStream_t st);
 int launch_attn_bwd(const AttnLaunch& L, cudaStream_t st);
+// Backward on tcgen05 (units of one head only; GSWA_ERR_UNSUPPORTED otherwise).
+int launch_attn_bwd_tc(const AttnLaunch& L, cudaStream_t st);
 
 // ---- orchestration
 bool fast_path_ok(const Plan& p);

@@ -652,19 +652,27 @@ size_t gt_smem_bytes(int natoms, int NB, int nstages) {
   return 1024 + (size_t)natoms * NB * 128 + (size_t)nstages * kAtomBytes + (size_t)128 * NB * 2 + (size_t)NB * 4 + 64;
 }
 
-int make_tmap(CUtensorMap* tm, const void* base, long long rows, int cols, int box_rows) {
-  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-  static EncodeFn fn = nullptr;
+typedef CUresult (*TmapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static TmapEncodeFn tmap_encoder() {
+  static TmapEncodeFn fn = nullptr;
   if (fn == nullptr) {
     void* p = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess || p == nullptr)
-      return check_launch() ? GSWA_ERR_CUDA : GSWA_ERR_CUDA;
-    fn = reinterpret_cast<EncodeFn>(p);
+        q != cudaDriverEntryPointSuccess || p == nullptr) {
+      (void)cudaGetLastError();
+      return nullptr;
+    }
+    fn = reinterpret_cast<TmapEncodeFn>(p);
   }
+  return fn;
+}
+
+int make_tmap(CUtensorMap* tm, const void* base, long long rows, int cols, int box_rows) {
+  const TmapEncodeFn fn = tmap_encoder();
+  if (fn == nullptr) return GSWA_ERR_CUDA;
   const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
   const cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
@@ -672,6 +680,20 @@ int make_tmap(CUtensorMap* tm, const void* base, long long rows, int cols, int b
   const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? GSWA_OK : GSWA_ERR_CUDA;
+}
+
+int make_tmap_window(CUtensorMap* tm, const void* base, long long img_rows, int W, int cols, int dp, int box_w, int box_h,
+                     bool swizzled) {
+  const TmapEncodeFn fn = tmap_encoder();
+  if (fn == nullptr) return GSWA_ERR_CUDA;
+  const cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)W, (cuuint64_t)img_rows};
+  const cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)cols * 2 * (cuuint64_t)W};
+  const cuuint32_t box[3] = {(cuuint32_t)dp, (cuuint32_t)box_w, (cuuint32_t)box_h};
+  const cuuint32_t es[3] = {1u, 1u, 1u};
+  const CUtensorMapSwizzle sw = !swizzled ? CU_TENSOR_MAP_SWIZZLE_NONE : (dp == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+  const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? GSWA_OK : GSWA_ERR_CUDA;
 }
 
