@@ -262,7 +262,7 @@ def run_ours(args, cfg):
     mem0 = torch.cuda.memory_allocated()
     torch.cuda.reset_peak_memory_stats()
     dev = {k: v.cuda() for k, v in host.items()}
-    desc = gb.Desc.from_config(cfg)
+    desc = gb.Desc.from_config(cfg, flags=args.flags)
     saved_b, fwd_b, infer_b, bwd_b = gb.gswa_workspace_query(desc)
     C, M, nh = cfg.C, cfg.window, cfg.num_heads
     y = torch.empty(inp["x"].shape, dtype=tdt, device="cuda")
@@ -385,7 +385,7 @@ def run_ours(args, cfg):
 
     line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic", "config": workload_config(cfg),
+            "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic", "config": dict(workload_config(cfg), flags=args.flags),
             "tflops": F * world / (ms_step * 1e-3) / 1e12,
             "layer_roofline": {"frac_burst": t_roof / (ms_step * 1e-3), "frac_sustained": t_roof_sus / (ms_step * 1e-3),
                                "roofline_us": t_roof * 1e6, "alg_flops": F, "alg_bytes": Bt, "peaks": pk_src},
@@ -467,6 +467,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="cM", choices=[k for k, c in CONFIGS.items() if c.backward])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--flags", type=int, default=0, help="GSWA_FLAG_* bits for the layer descriptor (measured alternatives: "
+                    "4 = fused QKV + forward attention, 8 = attention backward on tcgen05)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-checker timing leg")
     ap.add_argument("--no-unfused", action="store_true", help="skip the unfused memory baseline")
     args = ap.parse_args()

@@ -58,7 +58,7 @@ enum {
   GSWA_FLAG_ACCUMULATE = 1u, /* add into the parameter gradients instead of overwriting them */
   GSWA_FLAG_GENERIC = 2u,    /* force the shape-generic CUDA-core kernels (no tensor-core fast path) */
   GSWA_FLAG_FUSED_FWD = 4u,  /* tensor-core path: one kernel for QKV projection + forward attention (slower at C = 180; kept as a measured alternative) */
-  GSWA_FLAG_WARP_MMA_ATTN = 8u /* tensor-core path: attention backward with warp-level mma.sync instead of tcgen05 (the earlier kernel; kept as a measured alternative) */
+  GSWA_FLAG_TCGEN05_ATTN = 8u /* tensor-core path: attention backward on tcgen05 with TMEM accumulators instead of warp-level mma.sync (4 % slower at C = 180; kept as a measured alternative) */
 };
 
 /* Layer description (host memory, read during the call only). */

@@ -348,7 +348,7 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
   al.dtable = dtable; al.scale = 1.0f / sqrtf((float)p.d); al.err = err;
   bool one_head_units = true;
   for (int i = 0; i < al.nunits; ++i) one_head_units = one_head_units && al.u[i].nheads == 1;
-  if (one_head_units && !(p.flags & GSWA_FLAG_WARP_MMA_ATTN)) {
+  if (one_head_units && (p.flags & GSWA_FLAG_TCGEN05_ATTN)) {
     if ((rc = make_tmap_window(&al.tm_out, dqkv, (long long)p.B * p.H, p.W, 3 * p.Ap, p.dp, 8, 8, true))) return rc;
     // A window of a shifted group that wraps around the image edge is stored as four boxes.  Their shared-
     // memory sources must start on 128-byte boundaries, which an even shift guarantees; units with another

@@ -38,12 +38,14 @@ constexpr int kTcStages = 4;          // input ring: window pairs in flight
 constexpr int kTabPitch = 24;         // row pitch of the bias table in shared memory: the 32 lanes of a warp
                                       // (4 window rows x 8 window columns of queries) hit 32 different banks
 
-// Bounded waits of this kernel: the hardware suspends the waiting thread (see mbar_try_wait_suspend), so the
-// many warps that wait for the other group's turn cost the working warps nothing.
+// Bounded waits of this kernel: a non-blocking test followed by a short sleep.  A sleeping warp takes no issue
+// slots and no shared-memory bandwidth from the warps that work, and it notices the phase change within
+// the sleep time (a blocking try_wait was seen to come back several hundred nanoseconds late).
 __device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, volatile int* abort_s, int* err) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {               // each try suspends up to 1 us: far beyond any real wait
-    if (mbar_try_wait_suspend(bar, parity, 1000u)) return true;
-    if (*abort_s) return false;
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_test_wait(bar, parity)) return true;
+    __nanosleep(64);
+    if ((i & 63u) == 63u && *abort_s) return false;
   }
   *abort_s = 1;
   if (err) atomicExch(err, 1);
@@ -91,6 +93,12 @@ __device__ __forceinline__ void load_half(uint32_t taddr, float scale, uint32_t*
   if constexpr (DP == 32) tmem_ld16(taddr, v); else tmem_ld8(taddr, v);
   tmem_ld_wait();
 #pragma unroll
+  if (scale == 1.f) {       // resolved at compile time where the caller passes the literal
+#pragma unroll
+    for (int e = 0; e < DP / 4; ++e) w[e] = pack_bf16(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
+    return;
+  }
+#pragma unroll
   for (int e = 0; e < DP / 4; ++e) w[e] = pack_bf16(__uint_as_float(v[2 * e]) * scale, __uint_as_float(v[2 * e + 1]) * scale);
 }
 // ... stored to DP/2 consecutive elements of a padded token-major row,
@@ -135,7 +143,7 @@ __global__ void __maxnreg__(96) attn_bwd_tc_kernel(const __grid_constant__ AttnL
   float* tab = Ls + kTcStages * 128;                                  // [15][kTabPitch]
   float* hist = tab + 15 * kTabPitch;                                 // [225]
   float* Dx = hist + 228;                                             // [group][half][128] partial row sums
-  __shared__ uint64_t inFull[kTcStages], inEmpty[kTcStages], barS[2], barP[2], barO[2], barE[2], barFin;
+  __shared__ uint64_t inFull[kTcStages], inEmpty[kTcStages], barS[2], barP1[2], barP[2], barO1[2], barO[2], barE[2], barFin;
   __shared__ uint32_t tmem_s;
   __shared__ volatile int abort_s;
 
@@ -148,7 +156,7 @@ __global__ void __maxnreg__(96) attn_bwd_tc_kernel(const __grid_constant__ AttnL
   if (tid == 0) {
     abort_s = 0;
     for (int i = 0; i < kTcStages; ++i) { mbar_init(&inFull[i], 1); mbar_init(&inEmpty[i], 2); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&barS[i], 1); mbar_init(&barP[i], 8); mbar_init(&barO[i], 1); mbar_init(&barE[i], 2); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&barS[i], 1); mbar_init(&barP1[i], 8); mbar_init(&barO1[i], 1); mbar_init(&barP[i], 8); mbar_init(&barO[i], 1); mbar_init(&barE[i], 2); }
     mbar_init(&barFin, 1);
     mbar_init_fence();
   }
@@ -195,30 +203,38 @@ __global__ void __maxnreg__(96) attn_bwd_tc_kernel(const __grid_constant__ AttnL
       const uint64_t dP0 = make_desc(0, 8192, 1024);                    // [P_w0 | P_w1] or [dS_w0 | dS_w1], MN-major
       const uint64_t dQ0 = make_desc(0, 16, 1024);                      // dS_w0 over dS_w1 (128 rows), K-major
       constexpr int kStep = (16 * C::kRB) >> 4;                         // 16 rows of a tile
-      // The two rounds are issued in whatever order their inputs become ready: the second round of step mj as
-      // soon as its P and dS are written, the first round of step si as soon as its tiles have landed and the
-      // TMEM half of its group has been read out.  This one thread polls (it must watch two barriers at a time);
-      // all other waits of the kernel sleep.
-      int si = 0, mj = 0;
+      // Work is issued in whatever order its inputs become ready: dV of a step as soon as its P is written
+      // (while the softmax threads still compute dS), dK and dQ once dS is written, the first round of step si
+      // as soon as its tiles have landed and the TMEM half of its group has been read out.  This one thread
+      // polls without sleeping (it watches several barriers at a time).
+      int si = 0, vj = 0, mj = 0;
       uint32_t idle = 0;
       while (mj < nsteps) {
-        if (mj < si && mbar_test_wait(&barP[mj & 1], (mj >> 1) & 1)) {
-          // second round of step mj: dV, dK, dQ of both windows into the columns its scores occupied
+        if (mj < vj && mbar_test_wait(&barP[mj & 1], (mj >> 1) & 1)) {
+          // second round, part two, of step mj (dS is written, dP is read): dK and dQ of both windows
           fence_after_sync();
           const uint64_t sm0 = dM0 + (smem_u32(ring + (size_t)(mj % kTcStages) * C::kStage) >> 4);
           const uint64_t pb = smem_u32(ps + (size_t)(mj & 1) * C::kPS) >> 4;               // P_w0 | P_w1 | dS_w0 | dS_w1
           const uint32_t tO = tmem + (mj & 1) * 256;
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk)          // [dV_0 | dV_1] = [P_w0 | P_w1]^T [dO_w0 | dO_w1], 16 query rows per instruction
-            mma_bf16(tO, dP0 + pb + kk * 128, sm0 + ((6 * C::kTile) >> 4) + kk * kStep, idT, kk != 0);
-#pragma unroll
-          for (int kk = 0; kk < 4; ++kk)          // [dK_0 | dK_1] = [dS_w0 | dS_w1]^T [Q_w0 | Q_w1]
+          for (int kk = 0; kk < 4; ++kk)          // [dK_0 | dK_1] = [dS_w0 | dS_w1]^T [Q_w0 | Q_w1], 16 query rows per instruction
             mma_bf16(tO + 2 * DP, dP0 + pb + 1024 + kk * 128, sm0 + kk * kStep, idT, kk != 0);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)          // [dQ_0 | dQ_1] = [dS_w0 ; dS_w1] [K_w0 | K_w1], 16 keys per instruction
             mma_bf16(tO + 4 * DP, dQ0 + pb + 1024 + kk * 2, sm0 + ((2 * C::kTile) >> 4) + kk * kStep, idQ, kk != 0);
           commit(&barO[mj & 1]);
           ++mj;
+          idle = 0;
+        } else if (vj < si && mbar_test_wait(&barP1[vj & 1], (vj >> 1) & 1)) {
+          // second round, part one, of step vj (P is written, S is read): dV of both windows over the scores' columns
+          fence_after_sync();
+          const uint64_t sm0 = dM0 + (smem_u32(ring + (size_t)(vj % kTcStages) * C::kStage) >> 4);
+          const uint64_t pb = smem_u32(ps + (size_t)(vj & 1) * C::kPS) >> 4;
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)          // [dV_0 | dV_1] = [P_w0 | P_w1]^T [dO_w0 | dO_w1]
+            mma_bf16(tmem + (vj & 1) * 256, dP0 + pb + kk * 128, sm0 + ((6 * C::kTile) >> 4) + kk * kStep, idT, kk != 0);
+          commit(&barO1[vj & 1]);
+          ++vj;
           idle = 0;
         } else if (si < nsteps && mbar_test_wait(&inFull[si % kTcStages], (si / kTcStages) & 1) &&
                    (si < 2 || mbar_test_wait(&barE[si & 1], ((si >> 1) - 1) & 1))) {
@@ -234,9 +250,11 @@ __global__ void __maxnreg__(96) attn_bwd_tc_kernel(const __grid_constant__ AttnL
           commit(&barS[si & 1]);
           ++si;
           idle = 0;
-        } else if (++idle > kSpinLimit || abort_s) {
-          if (!abort_s) { abort_s = 1; if (L.err) atomicExch(L.err, 1); }
-          break;
+        } else {
+          if (++idle > kSpinLimit || abort_s) {
+            if (!abort_s) { abort_s = 1; if (L.err) atomicExch(L.err, 1); }
+            break;
+          }
         }
       }
       // nothing may still be running on the tensor core when TMEM is given back
@@ -326,6 +344,11 @@ __global__ void __maxnreg__(96) attn_bwd_tc_kernel(const __grid_constant__ AttnL
         }
         *dpart = D;
       }
+      // P is written and S is read: dV may run (it overwrites the scores' first columns)
+      fence_proxy_async();
+      fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&barP1[grp]);
       ok = bar_vote(pair_id, 64, ok);                      // the two warps that share these rows
       if (ok && valid) {
         D += *dpeer;
@@ -356,41 +379,48 @@ __global__ void __maxnreg__(96) attn_bwd_tc_kernel(const __grid_constant__ AttnL
         mbar_arrive(&inEmpty[pending]);
         pending = -1;
       }
-      // P and dS are written, S and dP are read: the second round may run (it overwrites S and dP)
+      // dS is written and dP is read: dK and dQ may run (dQ overwrites dP)
       fence_proxy_async();
       fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&barP[grp]);
 
+      // The step's input tiles are dead by the time their products are done and serve as staging for the output
+      // tiles (dQ over Q, dK over K, dV over V).  A window that lies inside the image is a box of the
+      // token-major buffer: one tiled bulk store per tile.  A window that wraps around the image edge (exactly
+      // the masked ones) goes out as four boxes (even shifts) or row by row.  Each thread moves half of its
+      // row's DP columns.  dV is ready first (it only needed P) and is drained while dK and dQ still run.
+      unsigned char* stg = ring + (size_t)slot * C::kStage + x * C::kTile;
+      long long tokrow = 0;
+      if (wmasked && !wrap_tma) {
+        int ti = wi * 8 + qa + u.s, tj = wj * 8 + qc + u.s;            // undo the cyclic shift
+        if (ti >= g.H) ti -= g.H;
+        if (tj >= g.W) tj -= g.W;
+        tokrow = ((long long)b * g.H + ti) * g.W + tj;
+      }
+      unsigned char* drow = reinterpret_cast<unsigned char*>(L.dqkv + tokrow * 3 * Ap + u.h0 * DP) + half * DP;
+      ok = ok && tc_wait_warp(&barO1[grp], n & 1, &abort_s, L.err);
+      fence_after_sync();
+      if (ok && valid) {
+        if (!wmasked) stage_half<DP>(tO + x * DP, 1.f, stg + 4 * C::kTile, q, half);
+        else if (wrap_tma) stage_half_linear<DP>(tO + x * DP, 1.f, stg + 4 * C::kTile + wrow * C::kRB + half * DP);
+        else store_half<DP>(tO + x * DP, 1.f, drow + Ap * 4);
+      }
       ok = ok && tc_wait_warp(&barO[grp], n & 1, &abort_s, L.err);
       fence_after_sync();
-      // The step's input tiles are dead now and serve as staging for the output tiles (dQ over Q, dK over K,
-      // dV over V).  A window that lies inside the image is a box of the token-major buffer: one tiled bulk
-      // store per tile.  A window that wraps around the image edge (exactly the masked ones) is stored row by
-      // row.  Each thread moves half of its row's DP columns.
-      unsigned char* stg = ring + (size_t)slot * C::kStage + x * C::kTile;
       if (ok && valid) {
+        // q was stored scaled by log2(e) (the scores live in the log2 domain): dK = dS^T q takes it back out
         if (!wmasked) {
           stage_half<DP>(tO + (4 + x) * DP, L.scale, stg, q, half);
-          // q was stored scaled by log2(e) (the scores live in the log2 domain): dK = dS^T q takes it back out
           stage_half<DP>(tO + (2 + x) * DP, kLn2, stg + 2 * C::kTile, q, half);
-          stage_half<DP>(tO + x * DP, 1.f, stg + 4 * C::kTile, q, half);
-          fence_proxy_async();
         } else if (wrap_tma) {
           stage_half_linear<DP>(tO + (4 + x) * DP, L.scale, stg + wrow * C::kRB + half * DP);
           stage_half_linear<DP>(tO + (2 + x) * DP, kLn2, stg + 2 * C::kTile + wrow * C::kRB + half * DP);
-          stage_half_linear<DP>(tO + x * DP, 1.f, stg + 4 * C::kTile + wrow * C::kRB + half * DP);
-          fence_proxy_async();
         } else {
-          int ti = wi * 8 + qa + u.s, tj = wj * 8 + qc + u.s;          // undo the cyclic shift
-          if (ti >= g.H) ti -= g.H;
-          if (tj >= g.W) tj -= g.W;
-          const long long tokrow = ((long long)b * g.H + ti) * g.W + tj;
-          unsigned char* drow = reinterpret_cast<unsigned char*>(L.dqkv + tokrow * 3 * Ap + u.h0 * DP) + half * DP;
           store_half<DP>(tO + (4 + x) * DP, L.scale, drow);
           store_half<DP>(tO + (2 + x) * DP, kLn2, drow + Ap * 2);
-          store_half<DP>(tO + x * DP, 1.f, drow + Ap * 4);
         }
+        fence_proxy_async();
       }
       fence_before_sync();
       if (!bar_vote(win_id, 128, ok)) break;               // the four warps of this window

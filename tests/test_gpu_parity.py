@@ -111,6 +111,7 @@ def test_random_shapes_tensor_core_path(cfg):
     ref = run_oracle(cfg, inp)
     assert_close(run_gpu(cfg, inp), ref, cfg.dtype)
     assert_close(run_gpu(cfg, inp, flags=gb.FLAG_FUSED_FWD), ref, cfg.dtype)
+    assert_close(run_gpu(cfg, inp, flags=gb.FLAG_TCGEN05_ATTN), ref, cfg.dtype)
 
 
 @pytest.mark.parametrize("cfg", [SWEEP[2], SWEEP[7], SWEEP[8]], ids=["f32", "bf16-c60", "bf16-c180"])
@@ -130,6 +131,26 @@ def test_fused_forward_kernel(cfg):
     assert_close(got, ref, cfg.dtype)
     inf = run_gpu(cfg, inp, flags=gb.FLAG_FUSED_FWD, inference=True)
     assert rel_err(inf["y"], got["y"]) == 0.0
+
+
+@pytest.mark.parametrize("cfg", [SWEEP[6], SWEEP[7], SWEEP[8], SWEEP[9], SWEEP[10]],
+                         ids=["c60", "c180", "uneven-groups-odd-shift", "one-group", "two-heads-odd-window-count"])
+def test_tcgen05_attention_backward(cfg):
+    """The opt-in attention backward on tcgen05 (window pairs, TMEM accumulators, tiled bulk stores): windows inside
+    the image, windows that wrap around its edge (even shift: four boxes; odd shift: row by row), an odd number
+    of windows (the last pair holds one window), both padded head widths."""
+    inp = make_inputs(cfg)
+    got = run_gpu(cfg, inp, flags=gb.FLAG_TCGEN05_ATTN)
+    ref = run_oracle(cfg, inp)
+    assert_close(got, ref, cfg.dtype)
+
+
+def test_tcgen05_attention_backward_training_shape():
+    cfg = CONFIGS["c3"]
+    inp = make_inputs(cfg, batch=3)
+    got = run_gpu(cfg, inp, flags=gb.FLAG_TCGEN05_ATTN)
+    ref = run_oracle(cfg, inp, chunk=3)
+    assert_close(got, ref, cfg.dtype)
 
 
 def test_null_biases_inference_mode_and_accumulate():
