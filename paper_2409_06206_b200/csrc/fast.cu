@@ -19,7 +19,7 @@ struct Unit {
 };
 
 struct TokenSplit {
-  int nsplit, NB, nstages, natoms;
+  int nsplit, NB, nstages, natoms, stream_b;
 };
 
 // Largest number of heads per work unit such that the QKV weight image, two activation stages and
@@ -51,6 +51,18 @@ int make_units(const Plan& p, Unit* units) {
 // the staging tile and at least three ring stages fit.
 bool token_split(int C, int K, TokenSplit* ts) {
   const int natoms = (K + 63) / 64;
+  {
+    // all output columns in one CTA: with the weight image resident if it fits, else streamed through the ring
+    const int NB = (int)align_up((size_t)C, 32);
+    const size_t fixed = 1024 + (size_t)128 * NB * 2 + NB * 4 + 64;
+    const size_t resident = (size_t)natoms * NB * 128, stage = 16384 + (size_t)NB * 128;
+    if (NB <= 256 && fixed + resident + 4 * 16384 > kSmemBudget && fixed + 4 * stage <= kSmemBudget) {
+      int S = (int)((kSmemBudget - fixed) / stage);
+      if (S > 8) S = 8;
+      *ts = TokenSplit{1, NB, S, natoms, 1};
+      return true;
+    }
+  }
   for (int nsplit = 1; nsplit <= kMaxUnits; nsplit *= 2) {
     const int NB = (int)align_up((size_t)(C + nsplit - 1) / nsplit, 32);
     if (NB > 256) continue;
@@ -58,7 +70,7 @@ bool token_split(int C, int K, TokenSplit* ts) {
     if (fixed + 4 * 16384 > kSmemBudget) continue;
     int S = (int)((kSmemBudget - fixed) / 16384);
     if (S > 8) S = 8;
-    *ts = TokenSplit{(C + NB - 1) / NB, NB, S, natoms};
+    *ts = TokenSplit{(C + NB - 1) / NB, NB, S, natoms, 0};
     return true;
   }
   return false;
@@ -266,7 +278,7 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
   GTLaunch gt{};
   if ((rc = make_tmap(&gt.tmA, A, p.T, p.Ap, 128))) return rc;
   gt.natoms = tp.natoms; gt.rows = p.T;
-  gt.out = (bf*)y; gt.ldo = p.C; gt.NB = tp.NB; gt.nstages = tp.nstages; gt.err = err;
+  gt.out = (bf*)y; gt.ldo = p.C; gt.NB = tp.NB; gt.nstages = tp.nstages; gt.stream_b = tp.stream_b; gt.err = err;
   for (int i = 0; i < tp.nsplit; ++i) {
     const int col0 = i * tp.NB;
     gt.s[i] = GTSplit{(const unsigned char*)sc + fs.pimg[i], (const float*)(sc + fs.pbias[i]), col0,
@@ -369,7 +381,7 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
     GTLaunch gt{};
     if ((rc = make_tmap(&gt.tmA, dqkv, p.T, 3 * p.Ap, 128))) return rc;
     gt.natoms = tx.natoms; gt.rows = p.T;
-    gt.out = (bf*)dx; gt.ldo = p.C; gt.NB = tx.NB; gt.nstages = tx.nstages; gt.err = err;
+    gt.out = (bf*)dx; gt.ldo = p.C; gt.NB = tx.NB; gt.nstages = tx.nstages; gt.stream_b = tx.stream_b; gt.err = err;
     for (int i = 0; i < tx.nsplit; ++i) {
       const int col0 = i * tx.NB;
       gt.s[i] = GTSplit{(const unsigned char*)sc + bs.ximg[i], nullptr, col0, (p.C - col0 < tx.NB ? p.C - col0 : tx.NB)};

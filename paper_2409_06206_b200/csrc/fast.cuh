@@ -80,6 +80,7 @@ struct GTLaunch {
   int ldo;
   int NB;                      // accumulator columns per CTA (multiple of 32, <= 256)
   int nstages;
+  int stream_b;                // 1: the weight image travels through the ring with the A atoms (see gt_kernel)
   GTSplit s[kMaxUnits];
   int* err;
 };

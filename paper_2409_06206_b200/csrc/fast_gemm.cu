@@ -243,17 +243,24 @@ __global__ void __launch_bounds__(kThreads2, 1) gt_kernel(const __grid_constant_
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = align1024(smem_raw);
   const int NB = L.NB, natoms = L.natoms, S = L.nstages;
+  // The B operand (weight image) either stays resident in shared memory, or - when all its K atoms do not
+  // fit beside the ring - travels through the ring with the A atoms: the image is small and lives in L2,
+  // so streaming it costs no HBM traffic, whereas splitting N over several CTAs would make every one of
+  // them read all of A.
+  const bool stream = L.stream_b != 0;
+  const int stage_bytes = kAtomBytes + (stream ? NB * 128 : 0);
   unsigned char* sB = sm;
-  unsigned char* ring = sB + (size_t)natoms * NB * 128;
-  unsigned char* stg = ring + (size_t)S * kAtomBytes;
+  unsigned char* ring = sB + (stream ? 0 : (size_t)natoms * NB * 128);
+  unsigned char* stg = ring + (size_t)S * stage_bytes;
   float* sBias = reinterpret_cast<float*>(stg + (size_t)128 * NB * 2);
   __shared__ uint64_t full[8], empty[8], tfull[2], tempty[2];
   __shared__ uint32_t tmem_s;
   __shared__ int abort_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  for (int i = tid; i < natoms * NB * 8; i += kThreads2)
-    reinterpret_cast<uint4*>(sB)[i] = __ldg(reinterpret_cast<const uint4*>(sp.Bimg) + i);
+  if (!stream)
+    for (int i = tid; i < natoms * NB * 8; i += kThreads2)
+      reinterpret_cast<uint4*>(sB)[i] = __ldg(reinterpret_cast<const uint4*>(sp.Bimg) + i);
   for (int i = tid; i < NB; i += kThreads2) sBias[i] = sp.bias ? sp.bias[i] : 0.f;
   fence_proxy_async();
   if (tid == 0) {
@@ -281,8 +288,10 @@ __global__ void __launch_bounds__(kThreads2, 1) gt_kernel(const __grid_constant_
       for (long long tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         for (int atom = 0; atom < natoms; ++atom) {
           if (!wait_bar(&empty[rp.slot], rp.ph ^ 1, &abort_s, L.err)) { ok = false; break; }
-          mbar_arrive_expect_tx(&full[rp.slot], kAtomBytes);
-          tma_load_2d(ringA + rp.slot * kAtomBytes, &L.tmA, atom * 64, (int)(tile * 128), &full[rp.slot]);
+          mbar_arrive_expect_tx(&full[rp.slot], (uint32_t)stage_bytes);
+          tma_load_2d(ringA + rp.slot * stage_bytes, &L.tmA, atom * 64, (int)(tile * 128), &full[rp.slot]);
+          if (stream)
+            bulk_load(ringA + rp.slot * stage_bytes + kAtomBytes, sp.Bimg + (size_t)atom * NB * 128, (uint32_t)NB * 128u, &full[rp.slot]);
           rp.advance(1, S);
         }
       }
@@ -302,8 +311,8 @@ __global__ void __launch_bounds__(kThreads2, 1) gt_kernel(const __grid_constant_
         for (int atom = 0; atom < natoms; ++atom) {
           if (!wait_bar(&full[rp.slot], rp.ph, &abort_s, L.err)) { ok = false; break; }
           fence_after_sync();
-          const uint64_t ad = a0 + (uint64_t)((rp.slot * kAtomBytes) >> 4);
-          const uint64_t bd = b0 + (uint64_t)((atom * NB * 128) >> 4);
+          const uint64_t ad = a0 + (uint64_t)((rp.slot * stage_bytes) >> 4);
+          const uint64_t bd = stream ? ad + (kAtomBytes >> 4) : b0 + (uint64_t)((atom * NB * 128) >> 4);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) mma_bf16(tmem + buf * NB, ad + 2 * kk, bd + 2 * kk, idesc, (atom | kk) != 0);
           commit(&empty[rp.slot]);
@@ -648,8 +657,9 @@ int launch_gw(const GWLaunch& L, int nunits, int Cp, int dp, cudaStream_t st, co
   return GSWA_ERR_UNSUPPORTED;
 }
 
-size_t gt_smem_bytes(int natoms, int NB, int nstages) {
-  return 1024 + (size_t)natoms * NB * 128 + (size_t)nstages * kAtomBytes + (size_t)128 * NB * 2 + (size_t)NB * 4 + 64;
+size_t gt_smem_bytes(int natoms, int NB, int nstages, int stream_b) {
+  return 1024 + (stream_b ? 0 : (size_t)natoms * NB * 128) + (size_t)nstages * (kAtomBytes + (stream_b ? (size_t)NB * 128 : 0)) +
+         (size_t)128 * NB * 2 + (size_t)NB * 4 + 64;
 }
 
 typedef CUresult (*TmapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -698,7 +708,7 @@ int make_tmap_window(CUtensorMap* tm, const void* base, long long img_rows, int 
 }
 
 int launch_gt(const GTLaunch& L, int nsplits, cudaStream_t st, const char* name) {
-  const size_t smem = gt_smem_bytes(L.natoms, L.NB, L.nstages);
+  const size_t smem = gt_smem_bytes(L.natoms, L.NB, L.nstages, L.stream_b);
   if (cudaFuncSetAttribute(gt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return check_launch();
   const long long n_tiles = (L.rows + 127) / 128;
