@@ -99,6 +99,24 @@ struct BwdScratch {
   size_t dO, dqkv, img[kMaxUnits], ximg[kMaxUnits], dummy, total;
 };
 
+int np_cols(int C) { return (int)align_up((size_t)C + 1, 64); }
+
+// Extents of the two weight-gradient GEMM launches (dW_proj: which = 0, dW_qkv: which = 1).
+struct GrShape {
+  int M, NP, mbpc, nsplit;
+};
+GrShape gr_shape(const Plan& p, int which) {
+  GrShape g{};
+  g.M = which ? 3 * p.Ap : p.C;
+  g.NP = which ? np_cols(p.C) : (int)align_up((size_t)p.Ap, 64);
+  // dW_qkv: x is copied once for two M blocks of dqkv; dW_proj: two M blocks per CTA measured slower (fewer TMA stages)
+  g.mbpc = which && 2 * g.NP <= 512 ? 2 : 1;
+  const int mblocks = ((g.M + 127) / 128 + g.mbpc - 1) / g.mbpc;
+  const long long ns = 148 / mblocks, cap = (p.T + 63) / 64;
+  g.nsplit = (int)(ns < cap ? (ns < 1 ? 1 : ns) : cap);
+  return g;
+}
+
 FwdScratch fwd_layout(const Plan& p, const Unit* units, int nu, const TokenSplit& ts) {
   FwdScratch s{};
   size_t off = 256;
@@ -130,8 +148,6 @@ BwdScratch bwd_layout(const Plan& p, const Unit* units, int nu, const TokenSplit
   s.total = off;
   return s;
 }
-
-int np_cols(int C) { return (int)align_up((size_t)C + 1, 64); }
 
 }  // namespace
 
@@ -319,19 +335,15 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
   int rc = launch_prep(jobs, nj, st);
   if (rc) return rc;
 
-  const int sms = 148;
   if (dw_proj || db_proj) {
     // dW^P = dy^T A (A fetched by TMA); db^P rides on the ones column of A when the head dim is padded
     GRLaunch gr{};
     if ((rc = make_tmap(&gr.tm, A, p.T, p.Ap, 64))) return rc;
     gr.tma_is_L = 0;
     gr.P = (const bf*)dy; gr.ldp = p.C; gr.pvalid = p.C;
-    gr.Ap = p.Ap; gr.dp = p.dp; gr.d = p.d; gr.C = p.C; gr.M = p.C; gr.rows = p.T;
-    gr.NP = (int)align_up((size_t)p.Ap, 64);
-    gr.mbpc = 1;                                   // two M blocks per CTA measured slower here (fewer TMA stages)
-    const int mblocks = ((p.C + 127) / 128 + gr.mbpc - 1) / gr.mbpc;
-    long long ns = sms / mblocks, cap = (p.T + 63) / 64;
-    gr.nsplit = (int)(ns < cap ? (ns < 1 ? 1 : ns) : cap);
+    const GrShape gs = gr_shape(p, 0);
+    gr.Ap = p.Ap; gr.dp = p.dp; gr.d = p.d; gr.C = p.C; gr.M = gs.M; gr.rows = p.T;
+    gr.NP = gs.NP; gr.mbpc = gs.mbpc; gr.nsplit = gs.nsplit;
     gr.out = dw_proj ? dw_proj : dummy; gr.colsum = p.d < p.dp ? db_proj : nullptr; gr.err = err;
     if ((rc = launch_gr(gr, st, "dwproj_gemm"))) return rc;
     if (db_proj && p.d == p.dp && (rc = launch_colsum_bf16((const bf*)dy, p.T, p.C, p.C, db_proj, st))) return rc;
@@ -394,12 +406,9 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
     if ((rc = make_tmap(&gr.tm, dqkv, p.T, 3 * p.Ap, 64))) return rc;
     gr.tma_is_L = 1;
     gr.P = (const bf*)x; gr.ldp = p.C; gr.pvalid = p.C;
-    gr.Ap = p.Ap; gr.dp = p.dp; gr.d = p.d; gr.C = p.C; gr.M = 3 * p.Ap; gr.rows = p.T;
-    gr.NP = np_cols(p.C);
-    gr.mbpc = 2 * gr.NP <= 512 ? 2 : 1;            // x is copied once for two M blocks of dqkv
-    const int mblocks = ((3 * p.Ap + 127) / 128 + gr.mbpc - 1) / gr.mbpc;
-    long long ns = sms / mblocks, cap = (p.T + 63) / 64;
-    gr.nsplit = (int)(ns < cap ? (ns < 1 ? 1 : ns) : cap);
+    const GrShape gs = gr_shape(p, 1);
+    gr.Ap = p.Ap; gr.dp = p.dp; gr.d = p.d; gr.C = p.C; gr.M = gs.M; gr.rows = p.T;
+    gr.NP = gs.NP; gr.mbpc = gs.mbpc; gr.nsplit = gs.nsplit;
     gr.out = dw_qkv ? dw_qkv : dummy; gr.colsum = db_qkv; gr.err = err;
     if ((rc = launch_gr(gr, st, "dwqkv_gemm"))) return rc;
   }

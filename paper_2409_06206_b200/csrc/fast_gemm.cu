@@ -380,6 +380,9 @@ __global__ void __launch_bounds__(kThreads2, 1) gt_kernel(const __grid_constant_
 // ==========================================================================================
 // gr_kernel
 // ==========================================================================================
+__device__ __forceinline__ void red_add_f32(float* p, float a) {
+  asm volatile("red.relaxed.gpu.global.add.f32 [%0], %1;" ::"l"(p), "f"(a) : "memory");
+}
 __device__ __forceinline__ void red_add_v2(float* p, float a, float b) {
   asm volatile("red.relaxed.gpu.global.add.v2.f32 [%0], {%1, %2};" ::"l"(p), "f"(a), "f"(b) : "memory");
 }
@@ -404,6 +407,7 @@ __global__ void __launch_bounds__(kThreadsR, 1) gr_kernel(const __grid_constant_
   unsigned char* ringT = sm;
   unsigned char* ringC = sm + (size_t)ST * tbytes;
   __shared__ uint64_t fullT[8], emptyT[8], fullC[kSets], emptyC[kSets], done;
+  __shared__ int rowmap[256], colmap[256];
   __shared__ uint32_t tmem_s;
   __shared__ int abort_s;
 
@@ -523,29 +527,43 @@ __global__ void __launch_bounds__(kThreadsR, 1) gr_kernel(const __grid_constant_
       if (ok) commit(&done);
     }
   } else {
+    // caller indices of this CTA's accumulator rows and columns (-1: padding, -2: the ones column)
+    {
+      const int ones = L.tma_is_L ? L.pvalid : (L.d < L.dp ? L.d : -1);
+      for (int i = tid; i < MB * 128; i += kEpiWarps * 32) {
+        const int mi = mb * 128 + i;
+        rowmap[i] = L.tma_is_L ? (mi < L.M ? unpad_index(mi, L.Ap, L.dp, L.d, L.C) : -1) : (mi < L.M ? mi : -1);
+      }
+      for (int ni = tid; ni < NP; ni += kEpiWarps * 32)
+        colmap[ni] = ni == ones ? -2 : (L.tma_is_L ? (ni < L.C ? ni : -1) : (ni < L.Ap ? unpad_index(ni, L.Ap, L.dp, L.d, L.C) : -1));
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+    }
     if (wait_bar_warp(&done, 0, &abort_s, L.err)) {
       fence_after_sync();
-      const int ones = L.tma_is_L ? L.pvalid : (L.d < L.dp ? L.d : -1);   // N index of the ones column
-      for (int blk = 0; blk < MB; ++blk)
-      for (int c0 = 0; c0 < NP; c0 += 32) {
-        const int mi = (mb + blk) * 128 + tid;                          // index in the M space
-        const int m = L.tma_is_L ? (mi < L.M ? unpad_index(mi, L.Ap, L.dp, L.d, L.C) : -1) : (mi < L.M ? mi : -1);
-        uint32_t v[32];
-        tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + blk * NP + c0, v);
-        tmem_ld_wait();
-        if (m >= 0) {
-          float* orow = L.out + (long long)m * L.C;
+      {
+        // Atomic accumulation into the caller's gradients.  The padded row and column indices were turned into
+        // caller indices once, while the MMAs ran (rowmap, colmap); each 32 x 32 block goes through shared memory
+        // so that one instruction adds 32 consecutive columns of one row (one 128-byte transaction).
+        float* tp = reinterpret_cast<float*>(sm) + warp * 32 * 33;
+        for (int blk = 0; blk < MB; ++blk)
+          for (int c0 = 0; c0 < NP; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + blk * NP + c0, v);
+            tmem_ld_wait();
+            __syncwarp();
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            const int ni = c0 + j;
-            if (ni == ones) {
-              if (L.colsum != nullptr) atomicAdd(L.colsum + m, __uint_as_float(v[j]));
-            } else {
-              const int n = L.tma_is_L ? (ni + 1 < L.C ? ni : -1) : (ni < L.Ap ? unpad_index(ni, L.Ap, L.dp, L.d, L.C) : -1);
-              if (n >= 0) red_add_v2(orow + n, __uint_as_float(v[j]), __uint_as_float(v[j + 1]));
+            for (int j = 0; j < 32; ++j) tp[lane * 33 + j] = __uint_as_float(v[j]);
+            __syncwarp();
+            const int n = colmap[c0 + lane];
+#pragma unroll 8
+            for (int r = 0; r < 32; ++r) {
+              const int m = rowmap[blk * 128 + warp * 32 + r];
+              if (m < 0) continue;
+              const float val = tp[r * 33 + lane];
+              if (n >= 0) red_add_f32(L.out + (long long)m * L.C + n, val);
+              else if (n == -2 && L.colsum != nullptr) atomicAdd(L.colsum + m, val);
             }
           }
-        }
       }
     }
   }
