@@ -383,6 +383,9 @@ __global__ void __launch_bounds__(kThreads2, 1) gt_kernel(const __grid_constant_
 __device__ __forceinline__ void red_add_f32(float* p, float a) {
   asm volatile("red.relaxed.gpu.global.add.f32 [%0], %1;" ::"l"(p), "f"(a) : "memory");
 }
+__device__ __forceinline__ void red_add_v4(float* p, float4 v) {
+  asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
 __device__ __forceinline__ void red_add_v2(float* p, float a, float b) {
   asm volatile("red.relaxed.gpu.global.add.v2.f32 [%0], {%1, %2};" ::"l"(p), "f"(a), "f"(b) : "memory");
 }
@@ -543,8 +546,10 @@ __global__ void __launch_bounds__(kThreadsR, 1) gr_kernel(const __grid_constant_
       {
         // Atomic accumulation into the caller's gradients.  The padded row and column indices were turned into
         // caller indices once, while the MMAs ran (rowmap, colmap); each 32 x 32 block goes through shared memory
-        // so that one instruction adds 32 consecutive columns of one row (one 128-byte transaction).
-        float* tp = reinterpret_cast<float*>(sm) + warp * 32 * 33;
+        // so that eight lanes add the 32 consecutive columns of one row with 16-byte vector reductions (the L2
+        // atomic units, not DRAM, bound this tail: every CTA adds its whole accumulator into the same addresses).
+        float* tp = reinterpret_cast<float*>(sm) + warp * 32 * 36;
+        const int l8 = lane & 7, r4 = lane >> 3;              // 8 lanes x 4 columns cover a row's 32 columns; 4 rows per instruction
         for (int blk = 0; blk < MB; ++blk)
           for (int c0 = 0; c0 < NP; c0 += 32) {
             uint32_t v[32];
@@ -552,16 +557,35 @@ __global__ void __launch_bounds__(kThreadsR, 1) gr_kernel(const __grid_constant_
             tmem_ld_wait();
             __syncwarp();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) tp[lane * 33 + j] = __uint_as_float(v[j]);
+            for (int j = 0; j < 32; j += 4)
+              *reinterpret_cast<float4*>(tp + lane * 36 + j) =
+                  make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
             __syncwarp();
-            const int n = colmap[c0 + lane];
-#pragma unroll 8
-            for (int r = 0; r < 32; ++r) {
+            const int n0 = colmap[c0 + 4 * l8], n3 = colmap[c0 + 4 * l8 + 3];
+            const bool run4 = n0 >= 0 && n3 == n0 + 3;                               // four consecutive targets
+            const bool vec = run4 && ((L.C & 3) == 0) && ((n0 & 3) == 0);            // ... 16-byte aligned
+            const bool pair = run4 && ((L.C & 1) == 0) && ((n0 & 1) == 0);           // ... or at least 8-byte aligned
+#pragma unroll 4
+            for (int rr = 0; rr < 32; rr += 4) {
+              const int r = rr + r4;
               const int m = rowmap[blk * 128 + warp * 32 + r];
               if (m < 0) continue;
-              const float val = tp[r * 33 + lane];
-              if (n >= 0) red_add_f32(L.out + (long long)m * L.C + n, val);
-              else if (n == -2 && L.colsum != nullptr) atomicAdd(L.colsum + m, val);
+              const float4 val = *reinterpret_cast<const float4*>(tp + r * 36 + 4 * l8);
+              float* o = L.out + (long long)m * L.C;
+              if (vec) {
+                red_add_v4(o + n0, val);
+              } else if (pair) {
+                red_add_v2(o + n0, val.x, val.y);
+                red_add_v2(o + n0 + 2, val.z, val.w);
+              } else {
+                const float e[4] = {val.x, val.y, val.z, val.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  const int n = colmap[c0 + 4 * l8 + k];
+                  if (n >= 0) red_add_f32(o + n, e[k]);
+                  else if (n == -2 && L.colsum != nullptr) atomicAdd(L.colsum + m, e[k]);
+                }
+              }
             }
           }
       }
