@@ -24,9 +24,9 @@ struct TokenSplit {
 
 // Largest number of heads per work unit such that the QKV weight image, two activation stages and
 // the accumulators fit one SM.
-int heads_per_unit(int Cp, int dp) {
+int heads_per_unit(int Cp, int dp, int cap) {
   int best = 0;
-  for (int n = 1; n <= 3; ++n) {
+  for (int n = 1; n <= cap; ++n) {
     const size_t NT = (size_t)n * 3 * dp;
     const int slots = Cp / 64 + 1 > 4 ? Cp / 64 + 1 : 4;
     const size_t smem = 1024 + NT * Cp * 2 + 8 * 2 * 32 * dp * 2 + (size_t)slots * 128 * 128 + NT * 4 + 64;   // weights, staging, ring
@@ -35,8 +35,10 @@ int heads_per_unit(int Cp, int dp) {
   return best;
 }
 
-int make_units(const Plan& p, Unit* units) {
-  const int hpu = heads_per_unit(p.Cp, p.dp);
+// `cap` heads per unit at most: 2 for the QKV projection (two heads' 6*dp columns are one MMA and leave TMEM room for
+// two tiles, so the MMAs of the next tile overlap this tile's epilogue), 3 for dO = dy W^P (dp columns per head).
+int make_units(const Plan& p, Unit* units, int cap) {
+  const int hpu = heads_per_unit(p.Cp, p.dp, cap);
   if (hpu == 0) return -1;
   int n = 0;
   for (int g = 0; g < p.G; ++g)
@@ -161,7 +163,7 @@ bool fast_path_ok(const Plan& p) {
   q.Cp = (int)align_up((size_t)p.C, 64);
   q.Ap = p.nh * q.dp;
   Unit units[kMaxUnits];
-  if (make_units(q, units) <= 0) return false;
+  if (make_units(q, units, 2) <= 0 || make_units(q, units, 3) <= 0) return false;
   TokenSplit a, b;
   return token_split(p.C, q.Ap, &a) && token_split(p.C, 3 * q.Ap, &b);
 }
@@ -171,8 +173,8 @@ void fast_plan_sizes(Plan* p) {
   p->dp = p->d <= 16 ? 16 : 32;
   p->Cp = (int)align_up((size_t)p->C, 64);
   p->Ap = p->nh * p->dp;
-  Unit units[kMaxUnits];
-  const int nu = make_units(*p, units);
+  Unit units[kMaxUnits], bunits[kMaxUnits];
+  const int nu = make_units(*p, units, 2), bnu = make_units(*p, bunits, 3);
   TokenSplit tp, tx;
   token_split(p->C, p->Ap, &tp);
   token_split(p->C, 3 * p->Ap, &tx);
@@ -183,7 +185,7 @@ void fast_plan_sizes(Plan* p) {
   p->saved_bytes = p->off_L + align_up(T * p->nh * 4, 256);
   p->fwd_scratch = fwd_layout(*p, units, nu, tp).total;
   p->infer_scratch = p->fwd_scratch + p->saved_bytes;
-  p->bwd_scratch = bwd_layout(*p, units, nu, tx).total;
+  p->bwd_scratch = bwd_layout(*p, bunits, bnu, tx).total;
 }
 
 // Work units of the attention kernels: one head per CTA when the unit table has room for every head (more,
@@ -217,7 +219,7 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
                  cudaStream_t st) {
   using bf = __nv_bfloat16;
   Unit units[kMaxUnits];
-  const int nu = make_units(p, units);
+  const int nu = make_units(p, units, 2);
   TokenSplit tp;
   if (nu <= 0 || !token_split(p.C, p.Ap, &tp)) return GSWA_ERR_UNSUPPORTED;
   const FwdScratch fs = fwd_layout(p, units, nu, tp);
@@ -230,12 +232,14 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
   float* Lt = reinterpret_cast<float*>(sv + p.off_L);
   if (cudaMemsetAsync(err, 0, 256, st) != cudaSuccess) return check_launch();
 
+  // With a spare K column (C < Cp) the QKV bias rides in the weight image and meets a column of ones in the A operand.
+  const bool fold_bias = p.C < p.Cp && b_qkv != nullptr && !(p.flags & GSWA_FLAG_FUSED_FWD);
   PrepJob jobs[16];
   int nj = 0;
   for (int i = 0; i < nu; ++i)
     jobs[nj++] = PrepJob{PREP_QKV, (const bf*)w_qkv, (const bf*)b_qkv, (unsigned char*)sc + fs.img[i],
                          (float*)(sc + fs.bias[i]), p.C, p.d, p.dp, units[i].h0, units[i].nheads, 0,
-                         units[i].nheads * 3 * p.dp, p.Cp, p.Ap};
+                         units[i].nheads * 3 * p.dp, p.Cp, p.Ap, fold_bias ? 1 : 0};
   for (int i = 0; i < tp.nsplit; ++i)
     jobs[nj++] = PrepJob{PREP_PROJ, (const bf*)w_proj, (const bf*)b_proj, (unsigned char*)sc + fs.pimg[i],
                          (float*)(sc + fs.pbias[i]), p.C, p.d, p.dp, 0, 0, i * tp.NB, tp.NB, tp.natoms * 64, p.Ap};
@@ -276,10 +280,14 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
       w.A = (const bf*)x; w.lda = p.C; w.kvalid = p.C;
       w.H = p.H; w.W = p.W; w.s = p.gs[u.g]; w.nW = p.nW; w.nWw = p.nWw; w.n_windows = geo.n_windows;
       w.Bimg = (const unsigned char*)sc + fs.img[i];
-      w.bias = (const float*)(sc + fs.bias[i]);
+      w.bias = fold_bias || b_qkv == nullptr ? nullptr : (const float*)(sc + fs.bias[i]);
+      w.ones_col = fold_bias ? 1 : 0;
       w.out = qkv + geo.qkv_off[u.g] + (long long)(u.h0 - p.gh0[u.g]) * 3 * 64 * p.dp;
       w.win_stride = (long long)p.gh[u.g] * 3 * 64 * p.dp;
-      w.nchunks = u.nheads; w.cw = 3 * p.dp; w.q_every3 = 1;
+      // one accumulator chunk per unit when its columns fit one MMA (N <= 256), else one per head
+      if (u.nheads * 3 * p.dp <= 256) { w.nchunks = 1; w.cw = u.nheads * 3 * p.dp; }
+      else { w.nchunks = u.nheads; w.cw = 3 * p.dp; }
+      w.q_every3 = 1;
       w.qscale = qscale;
     }
     if ((rc = launch_gw(gw, nu, p.Cp, p.dp, st, "qkv_gemm"))) return rc;
@@ -308,7 +316,7 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
                   float* db_proj, float* dtable, void* scratch, cudaStream_t st) {
   using bf = __nv_bfloat16;
   Unit units[kMaxUnits];
-  const int nu = make_units(p, units);
+  const int nu = make_units(p, units, 3);
   TokenSplit tx;
   if (nu <= 0 || !token_split(p.C, 3 * p.Ap, &tx)) return GSWA_ERR_UNSUPPORTED;
   const BwdScratch bs = bwd_layout(p, units, nu, tx);

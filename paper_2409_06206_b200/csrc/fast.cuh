@@ -59,11 +59,13 @@ struct GWUnit {
   int nchunks, cw;             // NT = nchunks*cw accumulator columns; cw multiple of 16 and of DP
   int q_every3;                // 1: blocks with index % 3 == 0 are scaled by qscale
   float qscale;
+  int ones_col;                // 1: the loaders put a one into K column `kvalid` (the weight image carries the bias in that row)
 };
 struct GWLaunch {
   GWUnit u[kMaxUnits];
   int* err;
   int nslots;                  // ring slots of 16 KB (set by launch_gw)
+  int cta0[kMaxUnits + 1];     // first CTA of every unit (set by launch_gw)
 };
 
 // ---- token GEMM: A rows in token order, fetched by TMA from a padded [rows, K] buffer; packed rows out
@@ -157,6 +159,7 @@ struct PrepJob {
   int C, d, dp, h0, nheads;    // head range for the per-head modes
   int n0, NT, KP;              // first output row (PREP_PROJ / PREP_QKV_T), rows, padded K
   int Ap;                      // heads * dp: K of PREP_PROJ / PREP_QKV_T runs over padded (kind, head, c) indices
+  int fold_bias;               // PREP_QKV: write the bias into image row k == C (needs C < KP) instead of bias_out
 };
 int launch_prep(const PrepJob* jobs, int njobs, cudaStream_t st);
 

@@ -26,7 +26,11 @@ namespace {
 // ==========================================================================================
 template <int CP, int DP>
 __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant__ GWLaunch L) {
-  const GWUnit& u = L.u[blockIdx.y];
+  // CTAs cta0[i] .. cta0[i+1]-1 work on unit i (units get CTAs in proportion to their work)
+  int ui = 0;
+  while (ui + 1 < kMaxUnits && (int)blockIdx.x >= L.cta0[ui + 1]) ++ui;
+  const GWUnit& u = L.u[ui];
+  const int bx = (int)blockIdx.x - L.cta0[ui], gxu = L.cta0[ui + 1] - L.cta0[ui];
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = align1024(smem_raw);
   constexpr int NA = CP / 64;                  // K atoms per tile
@@ -77,7 +81,7 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
     rp.init(set, S);
     int g = set;                                 // ring step = tile iteration * NA + atom
     int it = 0;
-    for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+    for (long long tile = bx; tile < n_tiles; tile += gxu, ++it) {
       // the two windows of the pair: cyclic shift + partition are this address arithmetic.  Tile row
       // r = 64*half + 8*a + lw holds slot (a, lw) of window `half`; this thread owns lw = rq and rq + 4.
       const char* col0[2][2];
@@ -103,18 +107,26 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
         if (!wait_bar_warp(&empty[rp.slot], rp.ph ^ 1, &abort_s, L.err)) { ok = false; break; }
         const uint32_t dst = ringA + rp.slot * kAtomBytes;
         const bool cv = atom * 128 + ll.pc * 8 < u.kvalid * 2;      // inside the valid columns of a source row
+        if (cv) {
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const bool v = wv[half] && cv;
+          for (int half = 0; half < 2; ++half) {
+            const bool v = wv[half];
 #pragma unroll
-          for (int a8 = 0; a8 < 8; ++a8) {
-            int i = i0[half] + a8;
-            if (i >= u.H) i -= u.H;
-            const long long off = i * line_bytes + atom * 128;
-            const int k = 16 * half + 2 * a8;
-            cp_async8(dst + ll.dst(k), v ? col0[half][0] + off : srcA, v);
-            cp_async8(dst + ll.dst(k + 1), v ? col0[half][1] + off : srcA, v);
+            for (int a8 = 0; a8 < 8; ++a8) {
+              int i = i0[half] + a8;
+              if (i >= u.H) i -= u.H;
+              const long long off = i * line_bytes + atom * 128;
+              const int k = 16 * half + 2 * a8;
+              cp_async8(dst + ll.dst(k), v ? col0[half][0] + off : srcA, v);
+              cp_async8(dst + ll.dst(k + 1), v ? col0[half][1] + off : srcA, v);
+            }
           }
+        } else {
+          // K padding: zeros, except a one in column kvalid when the bias rides in the weight image's row kvalid
+          const uint32_t w0 = (u.ones_col && atom * 64 + ll.pc * 4 == u.kvalid) ? 0x3F80u : 0u;
+#pragma unroll
+          for (int k = 0; k < 32; ++k)
+            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(dst + ll.dst(k)), "r"(w0), "r"(0u) : "memory");
         }
         cp_async_commit();
         cp_async_wait(0);
@@ -135,7 +147,7 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
       rp.init(0, S);
       int q = 0, qph = 0, qlast = 0;                               // ring position of the next chunk and its phase
       bool ok = true;
-      for (long long tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (long long tile = bx; tile < n_tiles && ok; tile += gxu) {
         int slot_a[NA];
         for (int c = 0; c < u.nchunks && ok; ++c) {
           if (!wait_bar(&tempty[q], qph ^ 1, &abort_s, L.err)) { ok = false; break; }
@@ -173,7 +185,7 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
     const uint32_t mystgA = smem_u32(mystg);
     int nst = 0, q = 0, qph = 0;                  // q, qph: ring position of the next chunk and its phase
     bool ok = true;
-    for (long long tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+    for (long long tile = bx; tile < n_tiles && ok; tile += gxu) {
       const long long win = 2 * tile + (quad >> 1);
       const bool valid = win < u.n_windows;
       __nv_bfloat16* obase = u.out + win * u.win_stride + (quad & 1) * 32 * DP;
@@ -197,18 +209,42 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
             __syncwarp();
           }
           tmem_ld_wait();
-          const float sc = (u.q_every3 && gb % 3 == 0) ? u.qscale : 1.f;
           unsigned char* piece = mystg + buf * kPiece - (quad & 1) * kPiece;   // tile_off counts rows from the block start
+          const bool scaled = u.q_every3 && gb % 3 == 0;
+          if (u.bias != nullptr) {                 // bias added here (no spare K column to carry it)
+            const float sc = scaled ? u.qscale : 1.f;
 #pragma unroll
-          for (int j = 0; j < DP / 8; ++j) {
-            const float4 b0v = *reinterpret_cast<const float4*>(sBias + gb * DP + 8 * j);
-            const float4 b1v = *reinterpret_cast<const float4*>(sBias + gb * DP + 8 * j + 4);
-            uint4 o;
-            o.x = pack_bf16((__uint_as_float(v[8 * j]) + b0v.x) * sc, (__uint_as_float(v[8 * j + 1]) + b0v.y) * sc);
-            o.y = pack_bf16((__uint_as_float(v[8 * j + 2]) + b0v.z) * sc, (__uint_as_float(v[8 * j + 3]) + b0v.w) * sc);
-            o.z = pack_bf16((__uint_as_float(v[8 * j + 4]) + b1v.x) * sc, (__uint_as_float(v[8 * j + 5]) + b1v.y) * sc);
-            o.w = pack_bf16((__uint_as_float(v[8 * j + 6]) + b1v.z) * sc, (__uint_as_float(v[8 * j + 7]) + b1v.w) * sc);
-            *reinterpret_cast<uint4*>(piece + tile_off<DP>(row, j)) = o;
+            for (int j = 0; j < DP / 8; ++j) {
+              const float4 b0v = *reinterpret_cast<const float4*>(sBias + gb * DP + 8 * j);
+              const float4 b1v = *reinterpret_cast<const float4*>(sBias + gb * DP + 8 * j + 4);
+              uint4 o;
+              o.x = pack_bf16((__uint_as_float(v[8 * j]) + b0v.x) * sc, (__uint_as_float(v[8 * j + 1]) + b0v.y) * sc);
+              o.y = pack_bf16((__uint_as_float(v[8 * j + 2]) + b0v.z) * sc, (__uint_as_float(v[8 * j + 3]) + b0v.w) * sc);
+              o.z = pack_bf16((__uint_as_float(v[8 * j + 4]) + b1v.x) * sc, (__uint_as_float(v[8 * j + 5]) + b1v.y) * sc);
+              o.w = pack_bf16((__uint_as_float(v[8 * j + 6]) + b1v.z) * sc, (__uint_as_float(v[8 * j + 7]) + b1v.w) * sc);
+              *reinterpret_cast<uint4*>(piece + tile_off<DP>(row, j)) = o;
+            }
+          } else if (scaled) {
+            const float sc = u.qscale;
+#pragma unroll
+            for (int j = 0; j < DP / 8; ++j) {
+              uint4 o;
+              o.x = pack_bf16(__uint_as_float(v[8 * j]) * sc, __uint_as_float(v[8 * j + 1]) * sc);
+              o.y = pack_bf16(__uint_as_float(v[8 * j + 2]) * sc, __uint_as_float(v[8 * j + 3]) * sc);
+              o.z = pack_bf16(__uint_as_float(v[8 * j + 4]) * sc, __uint_as_float(v[8 * j + 5]) * sc);
+              o.w = pack_bf16(__uint_as_float(v[8 * j + 6]) * sc, __uint_as_float(v[8 * j + 7]) * sc);
+              *reinterpret_cast<uint4*>(piece + tile_off<DP>(row, j)) = o;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < DP / 8; ++j) {
+              uint4 o;
+              o.x = pack_bf16(__uint_as_float(v[8 * j]), __uint_as_float(v[8 * j + 1]));
+              o.y = pack_bf16(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3]));
+              o.z = pack_bf16(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5]));
+              o.w = pack_bf16(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7]));
+              *reinterpret_cast<uint4*>(piece + tile_off<DP>(row, j)) = o;
+            }
           }
           fence_proxy_async();                     // the bulk copy reads these stores through the async proxy
           __syncwarp();
@@ -616,6 +652,7 @@ __global__ void prep_kernel(const __grid_constant__ PrepJobs J) {
     if (p.mode == PREP_QKV) {            // row n = (head, q|k|v, c) of W_qkv; k = input channel
       const int blk = n / p.dp, c = n % p.dp, h = p.h0 + blk / 3, kind = blk % 3;
       if (c < p.d && k < C) val = __bfloat162float(p.W[(long long)(kind * C + h * p.d + c) * C + k]);
+      else if (c < p.d && k == C && p.fold_bias && p.b != nullptr) val = __bfloat162float(p.b[kind * C + h * p.d + c]);   // meets the ones column of the A operand
     } else if (p.mode == PREP_PROJ_T) {  // row n = (head, c) -> input channel of W_proj; k = output channel
       const int h = p.h0 + n / p.dp, c = n % p.dp;
       if (c < p.d && k < C) val = __bfloat162float(p.W[(long long)k * C + h * p.d + c]);
@@ -631,7 +668,7 @@ __global__ void prep_kernel(const __grid_constant__ PrepJobs J) {
         __float2bfloat16_rn(val);
     if (k == 0 && p.bias_out != nullptr) {
       float bv = 0.f;
-      if (p.b != nullptr) {
+      if (p.b != nullptr && !p.fold_bias) {
         if (p.mode == PREP_QKV) {
           const int blk = n / p.dp, c = n % p.dp, h = p.h0 + blk / 3, kind = blk % 3;
           if (c < p.d) bv = __bfloat162float(p.b[kind * C + h * p.d + c]);
@@ -684,10 +721,23 @@ static int launch_gw_t(const GWLaunch& L, int nunits, cudaStream_t st, const cha
     return check_launch();
   GWLaunch Lc = L;
   Lc.nslots = nslots;
-  long long gx = num_sms() / nunits;
-  if (gx < 1) gx = 1;
-  if (gx > max_tiles) gx = max_tiles;
-  { KernelScope ks_(name, st); gw_kernel<CP, DP><<<dim3((unsigned)gx, nunits), kThreads2, smem, st>>>(Lc); }
+  // One CTA per SM; a unit's share of them follows its work per tile (the loads and MMA issue every unit pays,
+  // plus an epilogue proportional to its columns), so that all units finish together.
+  double wsum = 0, w[kMaxUnits];
+  for (int i = 0; i < nunits; ++i) { w[i] = 160.0 + L.u[i].nchunks * L.u[i].cw; wsum += w[i]; }
+  const int total = num_sms() < nunits ? nunits : num_sms();
+  int given = 0;
+  Lc.cta0[0] = 0;
+  for (int i = 0; i < nunits; ++i) {
+    int c = i + 1 == nunits ? total - given : (int)(total * w[i] / wsum + 0.5);
+    const long long t = (L.u[i].n_windows + 1) / 2;
+    if (c < 1) c = 1;
+    if (c > t && t > 0) c = (int)t;
+    given += c;
+    Lc.cta0[i + 1] = given;
+  }
+  for (int i = nunits + 1; i <= kMaxUnits; ++i) Lc.cta0[i] = given;
+  { KernelScope ks_(name, st); gw_kernel<CP, DP><<<dim3((unsigned)given), kThreads2, smem, st>>>(Lc); }
   return check_launch();
 }
 
