@@ -642,43 +642,52 @@ struct PrepJobs {
   PrepJob j[16];
 };
 
-__global__ void prep_kernel(const __grid_constant__ PrepJobs J) {
+// Value of image element (row n, K index k) and of the bias that goes with row n.
+__device__ __forceinline__ float prep_value(const PrepJob& p, int n, int k, int ldp, int dmask) {
+  const int C = p.C;
+  if (p.mode == PREP_QKV) {            // row n = (head, q|k|v, c) of W_qkv; k = input channel
+    const int blk = n >> ldp, c = n & dmask, h = p.h0 + blk / 3, kind = blk % 3;
+    if (c < p.d && k < C) return __bfloat162float(p.W[(long long)(kind * C + h * p.d + c) * C + k]);
+    if (c < p.d && k == C && p.fold_bias && p.b != nullptr) return __bfloat162float(p.b[kind * C + h * p.d + c]);   // meets the ones column of the A operand
+  } else if (p.mode == PREP_PROJ_T) {  // row n = (head, c) -> input channel of W_proj; k = output channel
+    const int h = p.h0 + (n >> ldp), c = n & dmask;
+    if (c < p.d && k < C) return __bfloat162float(p.W[(long long)k * C + h * p.d + c]);
+  } else if (p.mode == PREP_PROJ) {    // row n = output channel n0+n of W_proj; k = padded (head, c) input index
+    const int h = k >> ldp, c = k & dmask;
+    if (p.n0 + n < C && k < p.Ap && c < p.d) return __bfloat162float(p.W[(long long)(p.n0 + n) * C + h * p.d + c]);
+  } else {                             // PREP_QKV_T: row n = input channel n0+n; k = padded (kind, head, c) row of W_qkv
+    const int kind = (k >= p.Ap) + (k >= 2 * p.Ap), rem = k - kind * p.Ap, h = rem >> ldp, c = rem & dmask;
+    if (p.n0 + n < C && k < 3 * p.Ap && c < p.d) return __bfloat162float(p.W[(long long)(kind * C + h * p.d + c) * C + p.n0 + n]);
+  }
+  return 0.f;
+}
+
+// Threads run along the index that is contiguous in the source weight (k for the plain images, n for the
+// transposed ones), blocks along the other; the padded head width is a power of two, so nothing divides per element.
+__global__ void __launch_bounds__(256) prep_kernel(const __grid_constant__ PrepJobs J) {
   const PrepJob& p = J.j[blockIdx.y];
-  const int total = p.NT * p.KP;
-  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
-    const int n = e / p.KP, k = e % p.KP;
-    float val = 0.f;
-    const int C = p.C;
-    if (p.mode == PREP_QKV) {            // row n = (head, q|k|v, c) of W_qkv; k = input channel
-      const int blk = n / p.dp, c = n % p.dp, h = p.h0 + blk / 3, kind = blk % 3;
-      if (c < p.d && k < C) val = __bfloat162float(p.W[(long long)(kind * C + h * p.d + c) * C + k]);
-      else if (c < p.d && k == C && p.fold_bias && p.b != nullptr) val = __bfloat162float(p.b[kind * C + h * p.d + c]);   // meets the ones column of the A operand
-    } else if (p.mode == PREP_PROJ_T) {  // row n = (head, c) -> input channel of W_proj; k = output channel
-      const int h = p.h0 + n / p.dp, c = n % p.dp;
-      if (c < p.d && k < C) val = __bfloat162float(p.W[(long long)k * C + h * p.d + c]);
-    } else if (p.mode == PREP_PROJ) {    // row n = output channel n0+n of W_proj; k = padded (head, c) input index
-      const int h = k / p.dp, c = k % p.dp;
-      if (p.n0 + n < C && k < p.Ap && c < p.d) val = __bfloat162float(p.W[(long long)(p.n0 + n) * C + h * p.d + c]);
-    } else {                             // PREP_QKV_T: row n = input channel n0+n; k = padded (kind, head, c) row of W_qkv
-      const int kind = k / p.Ap, rem = k % p.Ap, h = rem / p.dp, c = rem % p.dp;
-      if (p.n0 + n < C && kind < 3 && c < p.d)
-        val = __bfloat162float(p.W[(long long)(kind * C + h * p.d + c) * C + p.n0 + n]);
+  const int ldp = p.dp == 32 ? 5 : 4, dmask = p.dp - 1;
+  const bool transposed = p.mode == PREP_PROJ_T || p.mode == PREP_QKV_T;
+  const int nouter = transposed ? p.KP : p.NT, ninner = transposed ? p.NT : p.KP;
+  for (int o = blockIdx.x; o < nouter; o += gridDim.x)
+    for (int i = threadIdx.x; i < ninner; i += blockDim.x) {
+      const int n = transposed ? i : o, k = transposed ? o : i;
+      *reinterpret_cast<__nv_bfloat16*>(p.img + (size_t)(k >> 6) * p.NT * 128 + sw128_offset(n, k & 63)) =
+          __float2bfloat16_rn(prep_value(p, n, k, ldp, dmask));
     }
-    *reinterpret_cast<__nv_bfloat16*>(p.img + (size_t)(k >> 6) * p.NT * 128 + sw128_offset(n, k & 63)) =
-        __float2bfloat16_rn(val);
-    if (k == 0 && p.bias_out != nullptr) {
+  if (p.bias_out != nullptr)
+    for (int n = blockIdx.x * blockDim.x + threadIdx.x; n < p.NT; n += gridDim.x * blockDim.x) {
       float bv = 0.f;
       if (p.b != nullptr && !p.fold_bias) {
         if (p.mode == PREP_QKV) {
-          const int blk = n / p.dp, c = n % p.dp, h = p.h0 + blk / 3, kind = blk % 3;
-          if (c < p.d) bv = __bfloat162float(p.b[kind * C + h * p.d + c]);
+          const int blk = n >> ldp, c = n & dmask, h = p.h0 + blk / 3, kind = blk % 3;
+          if (c < p.d) bv = __bfloat162float(p.b[kind * p.C + h * p.d + c]);
         } else if (p.mode == PREP_PROJ) {
-          if (p.n0 + n < C) bv = __bfloat162float(p.b[p.n0 + n]);
+          if (p.n0 + n < p.C) bv = __bfloat162float(p.b[p.n0 + n]);
         }
       }
       p.bias_out[n] = bv;
     }
-  }
 }
 
 }  // namespace
@@ -688,7 +697,7 @@ int launch_prep(const PrepJob* jobs, int njobs, cudaStream_t st) {
   if (njobs > 16) return GSWA_ERR_UNSUPPORTED;
   PrepJobs J{};
   for (int i = 0; i < njobs; ++i) J.j[i] = jobs[i];
-  { KernelScope ks_("prep_weights", st); prep_kernel<<<dim3(64, njobs), 256, 0, st>>>(J); }
+  { KernelScope ks_("prep_weights", st); prep_kernel<<<dim3(96, njobs), 256, 0, st>>>(J); }
   return check_launch();
 }
 
