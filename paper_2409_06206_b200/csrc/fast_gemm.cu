@@ -58,9 +58,7 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
   }
   // TMEM holds a ring of RC accumulator chunks of cw columns; a tile takes nchunks consecutive ring
   // positions, so the MMAs of the next tile start while this tile's chunks are still being drained.
-  // (With several chunks per tile the overlap only makes the MMAs and the epilogue fight for shared-memory
-  // bandwidth -- measured slower -- so the ring is then exactly one tile deep.)
-  const int RC = u.nchunks > 1 ? u.nchunks : (512 / u.cw < 8 ? 512 / u.cw : 8);
+  const int RC = 512 / u.cw < 8 ? 512 / u.cw : 8;
   const uint32_t tcols = pow2_cols(RC * u.cw);
   if (warp == kEpi2) tmem_alloc(&tmem_s, tcols);
   fence_before_sync();
@@ -184,16 +182,23 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
     unsigned char* mystg = stg + (size_t)warp * 2 * kPiece;
     const uint32_t mystgA = smem_u32(mystg);
     int nst = 0, q = 0, qph = 0;                  // q, qph: ring position of the next chunk and its phase
+    // A tile's completion is signalled on the ring position of its LAST chunk only.  The last positions of
+    // successive tiles cycle with period RC / gcd(nchunks, RC) tiles and visit every position of the cycle once,
+    // so the barrier at a tile's last position has flipped (tile iteration / period) times before.
+    int gcd_ = u.nchunks, rem_ = RC;
+    while (rem_) { const int t_ = gcd_ % rem_; gcd_ = rem_; rem_ = t_; }
+    const int period = RC / gcd_;
+    int it = 0;
     bool ok = true;
-    for (long long tile = bx; tile < n_tiles && ok; tile += gxu) {
+    for (long long tile = bx; tile < n_tiles && ok; tile += gxu, ++it) {
       const long long win = 2 * tile + (quad >> 1);
       const bool valid = win < u.n_windows;
       __nv_bfloat16* obase = u.out + win * u.win_stride + (quad & 1) * 32 * DP;
       {
         // the tile is complete when its last chunk is (MMAs finish in issue order)
-        int ql = q + u.nchunks - 1, pl = qph;
-        if (ql >= RC) { ql -= RC; pl ^= 1; }
-        if (!wait_bar_warp(&tfull[ql], pl, &abort_s, L.err)) break;
+        int ql = q + u.nchunks - 1;
+        if (ql >= RC) ql -= RC;
+        if (!wait_bar_warp(&tfull[ql], (it / period) & 1, &abort_s, L.err)) break;
       }
       for (int c = 0; c < u.nchunks; ++c) {
         fence_after_sync();
