@@ -97,6 +97,7 @@ struct GRLaunch {
   int tma_is_L;
   const __nv_bfloat16* P;      // the copy-fed operand, [rows, ldp] with pvalid valid columns
   int ldp, pvalid;
+  int p16;                     // 16-byte copies possible for: 0 no row, 1 even rows, 2 all rows of P (set by launch_gr)
   int Ap, dp, d, C;
   int M;                       // extent of the M index space (3*Ap or C)
   long long rows;

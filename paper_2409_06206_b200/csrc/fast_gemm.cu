@@ -521,6 +521,8 @@ __global__ void __launch_bounds__(kThreadsR, 1) gr_kernel(const __grid_constant_
       }
     const char* const srcP = reinterpret_cast<const char*>(L.P);
     const long long prow = (long long)L.ldp * 2;
+    // rows of this thread that start on 16-byte boundaries: all of them, the even ones (its rows all have lw's parity), or none
+    const bool row16 = L.p16 == 2 || (L.p16 == 1 && (ll.lw & 1) == 0);
     const uint32_t sS = smem_u32(base);
     int ph = 0;
     for (int s = set; s < nst; s += kSets, ph ^= 1) {
@@ -537,8 +539,12 @@ __global__ void __launch_bounds__(kThreadsR, 1) gr_kernel(const __grid_constant_
         for (int k = 0; k < 8; ++k) {
           const bool tv = whole || tb + ll.lw + 8 * k < t1;
           const char* src = pp + k * 8 * prow + a * 128;
-          cp_async8(dst + k * 1024, tv ? src : srcP, tv);
-          if (v1) cp_async8(dst + k * 1024 + 8, tv ? src + 8 : srcP, tv);
+          if (row16 && v1) {
+            cp_async16(dst + k * 1024, tv ? src : srcP, tv);
+          } else {
+            cp_async8(dst + k * 1024, tv ? src : srcP, tv);
+            if (v1) cp_async8(dst + k * 1024 + 8, tv ? src + 8 : srcP, tv);
+          }
         }
       }
       cp_async_commit();
@@ -828,6 +834,8 @@ int launch_gt(const GTLaunch& L, int nsplits, cudaStream_t st, const char* name)
 int launch_gr(const GRLaunch& L, cudaStream_t st, const char* name) {
   GRLaunch Lc = L;
   if (Lc.mbpc < 1 || Lc.mbpc * L.NP > 512) Lc.mbpc = 1;
+  // 16-byte copies need 16-byte aligned sources: the base, and a row pitch of 0 (every row) or 8 (even rows) mod 16
+  Lc.p16 = (reinterpret_cast<uintptr_t>(L.P) & 15) != 0 ? 0 : ((L.ldp * 2) % 16 == 0 ? 2 : ((L.ldp * 2) % 16 == 8 ? 1 : 0));
   const int latoms = 2 * Lc.mbpc, ratoms = L.NP / 64;
   const size_t tbytes = (size_t)(L.tma_is_L ? latoms : ratoms) * 8192, cbytes = (size_t)(L.tma_is_L ? ratoms : latoms) * 8192;
   const size_t budget = 215 * 1024;

@@ -116,12 +116,14 @@ struct LoaderLane {
 };
 
 // Lane mapping of gr_kernel's copy-fed operand: rows lw + 8k, 16-byte chunk pp of the atom row (two
-// 8-byte pieces); a copy instruction reads four rows of 128 contiguous bytes.
+// 8-byte pieces); a copy instruction reads four rows of 128 contiguous bytes.  The first warp of a set takes
+// the even rows, the second the odd ones: with a row pitch of 8 mod 16 bytes the even rows start on 16-byte
+// boundaries and are fetched with half as many (16-byte) copies, and a warp never mixes the two kinds.
 struct LoaderLane4 {
   int lw, pp;
   uint32_t dst0;
   __device__ __forceinline__ void init(int ts) {
-    lw = ts >> 3;
+    lw = ((ts >> 3) & 3) * 2 + (ts >> 5);
     pp = ts & 7;
     dst0 = sw128_offset(lw, pp * 8);
   }
