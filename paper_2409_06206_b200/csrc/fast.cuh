@@ -59,6 +59,7 @@ struct GWUnit {
   int nchunks, cw;             // NT = nchunks*cw accumulator columns; cw multiple of 16 and of DP
   int q_every3;                // 1: blocks with index % 3 == 0 are scaled by qscale
   float qscale;
+  int a16;                     // 16-byte copies possible for: 0 no row, 1 rows of even tokens, 2 all rows of A (set by launch_gw)
   int ones_col;                // 1: the loaders put a one into K column `kvalid` (the weight image carries the bias in that row)
 };
 struct GWLaunch {

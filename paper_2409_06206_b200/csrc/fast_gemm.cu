@@ -74,6 +74,9 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
     ll.init(((warp - kEpi2 - 1) & 1) * 32 + lane);
     const char* const srcA = reinterpret_cast<const char*>(u.A);
     const long long row_bytes = (long long)u.lda * 2, line_bytes = (long long)u.W * row_bytes;
+    // Rows of this thread that start on 16-byte boundaries: all, or those of even tokens.  The token parity of tile
+    // row (a, c) is that of shift + c (image width and height are even), and c = rq or rq + 4 for all rows of a thread.
+    const bool row16 = u.a16 == 2 || (u.a16 == 1 && ((u.s + ll.rq) & 1) == 0);
     const uint32_t ringA = smem_u32(ring);
     RingPos rp;
     rp.init(set, S);
@@ -105,7 +108,25 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
         if (!wait_bar_warp(&empty[rp.slot], rp.ph ^ 1, &abort_s, L.err)) { ok = false; break; }
         const uint32_t dst = ringA + rp.slot * kAtomBytes;
         const bool cv = atom * 128 + ll.pc * 8 < u.kvalid * 2;      // inside the valid columns of a source row
-        if (cv) {
+        // rows on 16-byte boundaries: the even piece's thread copies both pieces of a fully valid 16-byte chunk
+        const bool c16 = row16 && atom * 128 + (ll.pc | 1) * 8 < u.kvalid * 2;
+        if (c16) {
+          if ((ll.pc & 1) == 0) {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              const bool v = wv[half];
+#pragma unroll
+              for (int a8 = 0; a8 < 8; ++a8) {
+                int i = i0[half] + a8;
+                if (i >= u.H) i -= u.H;
+                const long long off = i * line_bytes + atom * 128;
+                const int k = 16 * half + 2 * a8;
+                cp_async16(dst + ll.dst(k), v ? col0[half][0] + off : srcA, v);
+                cp_async16(dst + ll.dst(k + 1), v ? col0[half][1] + off : srcA, v);
+              }
+            }
+          }
+        } else if (cv) {
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
             const bool v = wv[half];
@@ -741,6 +762,10 @@ static int launch_gw_t(const GWLaunch& L, int nunits, cudaStream_t st, const cha
     return check_launch();
   GWLaunch Lc = L;
   Lc.nslots = nslots;
+  for (int i = 0; i < nunits; ++i) {      // 16-byte copies need 16-byte aligned sources (see the loaders)
+    const GWUnit& un = L.u[i];
+    Lc.u[i].a16 = (reinterpret_cast<uintptr_t>(un.A) & 15) != 0 || (un.W & 1) || (un.H & 1) ? 0 : ((un.lda * 2) % 16 == 0 ? 2 : ((un.lda * 2) % 16 == 8 ? 1 : 0));
+  }
   // One CTA per SM; a unit's share of them follows its work per tile (the loads and MMA issue every unit pays,
   // plus an epilogue proportional to its columns), so that all units finish together.
   double wsum = 0, w[kMaxUnits];

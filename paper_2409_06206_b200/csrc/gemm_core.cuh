@@ -102,12 +102,14 @@ struct RingPos {
 // rows rq + 4k (rq = 0..3).  Sixteen consecutive lanes cover one whole atom row: a copy instruction
 // reads two runs of 128 contiguous bytes and writes two full rows of shared memory (no bank
 // conflicts).  (r & 7) alternates between rq (k even) and rq + 4 (k odd), hence two swizzled bases;
-// the destination of row rq + 4k is base + 512 k.
+// the destination of row rq + 4k is base + 512 k.  The first warp of a set takes rq = 0 and 2, the second
+// rq = 1 and 3: all rows of a warp then have the same parity of their column in the window, hence of
+// their token index, and a warp can use 16-byte copies for all of them or for none.
 struct LoaderLane {
   int rq, pc;
   uint32_t dst_e, dst_o;
   __device__ __forceinline__ void init(int ts) {
-    rq = ts >> 4;
+    rq = ((ts >> 4) & 1) * 2 + (ts >> 5);
     pc = ts & 15;
     dst_e = sw128_offset(rq, pc * 4);
     dst_o = sw128_offset(rq + 4, pc * 4) - 4 * 128;
