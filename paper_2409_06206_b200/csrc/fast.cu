@@ -234,6 +234,8 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
 
   // With a spare K column (C < Cp) the QKV bias rides in the weight image and meets a column of ones in the A operand.
   const bool fold_bias = p.C < p.Cp && b_qkv != nullptr && !(p.flags & GSWA_FLAG_FUSED_FWD);
+  // Likewise the output projection's bias meets the ones that column d of head 0 of the attention output holds.
+  const bool fold_pbias = p.d < p.dp && b_proj != nullptr;
   PrepJob jobs[16];
   int nj = 0;
   for (int i = 0; i < nu; ++i)
@@ -242,7 +244,8 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
                          units[i].nheads * 3 * p.dp, p.Cp, p.Ap, fold_bias ? 1 : 0};
   for (int i = 0; i < tp.nsplit; ++i)
     jobs[nj++] = PrepJob{PREP_PROJ, (const bf*)w_proj, (const bf*)b_proj, (unsigned char*)sc + fs.pimg[i],
-                         (float*)(sc + fs.pbias[i]), p.C, p.d, p.dp, 0, 0, i * tp.NB, tp.NB, tp.natoms * 64, p.Ap};
+                         (float*)(sc + fs.pbias[i]), p.C, p.d, p.dp, 0, 0, i * tp.NB, tp.NB, tp.natoms * 64, p.Ap,
+                         fold_pbias ? 1 : 0};
   int rc = launch_prep(jobs, nj, st);
   if (rc) return rc;
 
@@ -305,7 +308,7 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
   gt.out = (bf*)y; gt.ldo = p.C; gt.NB = tp.NB; gt.nstages = tp.nstages; gt.stream_b = tp.stream_b; gt.err = err;
   for (int i = 0; i < tp.nsplit; ++i) {
     const int col0 = i * tp.NB;
-    gt.s[i] = GTSplit{(const unsigned char*)sc + fs.pimg[i], (const float*)(sc + fs.pbias[i]), col0,
+    gt.s[i] = GTSplit{(const unsigned char*)sc + fs.pimg[i], fold_pbias || b_proj == nullptr ? nullptr : (const float*)(sc + fs.pbias[i]), col0,
                       (p.C - col0 < tp.NB ? p.C - col0 : tp.NB)};
   }
   return launch_gt(gt, tp.nsplit, st, "proj_gemm");

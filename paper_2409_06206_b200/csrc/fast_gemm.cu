@@ -401,13 +401,21 @@ __global__ void __launch_bounds__(kThreads2, 1) gt_kernel(const __grid_constant_
         // the lane's row of the staging tile; rows are 2*ncols bytes apart (a multiple of 8, and an
         // odd multiple for C = 180, so these 8-byte stores do not collide on banks)
         uint2* dst = reinterpret_cast<uint2*>(mystg + ((size_t)lane * ncols + c0) * 2);
+        if (sp.bias != nullptr) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-          if (c0 + 4 * j < ncols) {
-            const float4 bq = *reinterpret_cast<const float4*>(sBias + c0 + 4 * j);
-            dst[j] = make_uint2(pack_bf16(__uint_as_float(v[4 * j]) + bq.x, __uint_as_float(v[4 * j + 1]) + bq.y),
-                                pack_bf16(__uint_as_float(v[4 * j + 2]) + bq.z, __uint_as_float(v[4 * j + 3]) + bq.w));
-          }
+          for (int j = 0; j < 8; ++j)
+            if (c0 + 4 * j < ncols) {
+              const float4 bq = *reinterpret_cast<const float4*>(sBias + c0 + 4 * j);
+              dst[j] = make_uint2(pack_bf16(__uint_as_float(v[4 * j]) + bq.x, __uint_as_float(v[4 * j + 1]) + bq.y),
+                                  pack_bf16(__uint_as_float(v[4 * j + 2]) + bq.z, __uint_as_float(v[4 * j + 3]) + bq.w));
+            }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (c0 + 4 * j < ncols)
+              dst[j] = make_uint2(pack_bf16(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1])),
+                                  pack_bf16(__uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
+        }
       }
       fence_before_sync();
       __syncwarp();
@@ -687,6 +695,7 @@ __device__ __forceinline__ float prep_value(const PrepJob& p, int n, int k, int 
   } else if (p.mode == PREP_PROJ) {    // row n = output channel n0+n of W_proj; k = padded (head, c) input index
     const int h = k >> ldp, c = k & dmask;
     if (p.n0 + n < C && k < p.Ap && c < p.d) return __bfloat162float(p.W[(long long)(p.n0 + n) * C + h * p.d + c]);
+    if (p.n0 + n < C && k == p.d && p.fold_bias && p.b != nullptr) return __bfloat162float(p.b[p.n0 + n]);   // meets the ones in column d of head 0 of A
   } else {                             // PREP_QKV_T: row n = input channel n0+n; k = padded (kind, head, c) row of W_qkv
     const int kind = (k >= p.Ap) + (k >= 2 * p.Ap), rem = k - kind * p.Ap, h = rem >> ldp, c = rem & dmask;
     if (p.n0 + n < C && k < 3 * p.Ap && c < p.d) return __bfloat162float(p.W[(long long)(kind * C + h * p.d + c) * C + p.n0 + n]);
