@@ -113,7 +113,9 @@ int gswa_forward_static(const gswa_desc* desc, const void* x, const void* w_qkv,
                         const void* w_proj, const void* b_proj, const void* bias_table, void* y, void* cuda_stream);
 
 /* Backward pass (reverse mode of gswa_forward; the paper's stated target is the memory of
- * back-propagation).  `saved` is the buffer written by gswa_forward for the same desc and inputs.
+ * back-propagation).  `saved` is the buffer written by gswa_forward for the same desc and inputs; the weights must
+ * be the ones that call was given (on the tensor-core path `saved` also carries the re-laid-out copies of them that
+ * the backward GEMMs read, so that this call launches no preparation kernel).
  * Writes dx (element type `dtype`) and the float32 parameter gradients dw_qkv[3C,C], db_qkv[3C],
  * dw_proj[C,C], db_proj[C], dbias_table[(2M-1)^2, num_heads]; each gradient pointer may be NULL to
  * skip it (dx included).  Gradients are overwritten unless GSWA_FLAG_ACCUMULATE is set.  Float32

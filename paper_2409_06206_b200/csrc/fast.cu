@@ -98,7 +98,12 @@ struct FwdScratch {
   size_t img[kMaxUnits], bias[kMaxUnits], pimg[kMaxUnits], pbias[kMaxUnits], total;
 };
 struct BwdScratch {
-  size_t dO, dqkv, img[kMaxUnits], ximg[kMaxUnits], dummy, total;
+  size_t dO, dqkv, dummy, total;
+};
+// Weight images of the backward GEMMs (W^P transposed per unit, W_qkv transposed per column split).  A training
+// forward call builds them next to its own images, into `saved`, so that the backward call launches no prep kernel.
+struct BwdImages {
+  size_t img[kMaxUnits], ximg[kMaxUnits], total;
 };
 
 int np_cols(int C) { return (int)align_up((size_t)C + 1, 64); }
@@ -135,17 +140,24 @@ FwdScratch fwd_layout(const Plan& p, const Unit* units, int nu, const TokenSplit
   return s;
 }
 
-BwdScratch bwd_layout(const Plan& p, const Unit* units, int nu, const TokenSplit& tx) {
-  BwdScratch s{};
-  size_t off = 256;
-  s.dO = off; off += align_up((size_t)p.T * p.nh * p.dp * 2, 256);
-  s.dqkv = off; off += align_up((size_t)p.T * 3 * p.Ap * 2, 256);
+BwdImages bwd_images(const Plan& p, const Unit* units, int nu, const TokenSplit& tx) {
+  BwdImages s{};
+  size_t off = 0;
   for (int i = 0; i < nu; ++i) {
     s.img[i] = off; off += align_up((size_t)units[i].nheads * p.dp * p.Cp * 2, 256);
   }
   for (int i = 0; i < tx.nsplit; ++i) {
     s.ximg[i] = off; off += align_up((size_t)tx.natoms * tx.NB * 128, 256);
   }
+  s.total = off;
+  return s;
+}
+
+BwdScratch bwd_layout(const Plan& p) {
+  BwdScratch s{};
+  size_t off = 256;
+  s.dO = off; off += align_up((size_t)p.T * p.nh * p.dp * 2, 256);
+  s.dqkv = off; off += align_up((size_t)p.T * 3 * p.Ap * 2, 256);
   s.dummy = off; off += align_up((size_t)3 * p.C * p.C * 4, 256);
   s.total = off;
   return s;
@@ -182,10 +194,11 @@ void fast_plan_sizes(Plan* p) {
   p->off_qkv = 0;
   p->off_A = align_up(T * 3 * p->nh * p->dp * 2, 256);
   p->off_L = p->off_A + align_up(T * p->Ap * 2, 256);
-  p->saved_bytes = p->off_L + align_up(T * p->nh * 4, 256);
+  p->off_bimg = p->off_L + align_up(T * p->nh * 4, 256);
+  p->saved_bytes = p->off_bimg + bwd_images(*p, bunits, bnu, tx).total;
   p->fwd_scratch = fwd_layout(*p, units, nu, tp).total;
   p->infer_scratch = p->fwd_scratch + p->saved_bytes;
-  p->bwd_scratch = bwd_layout(*p, bunits, bnu, tx).total;
+  p->bwd_scratch = bwd_layout(*p).total;
 }
 
 // Work units of the attention kernels: one head per CTA when the unit table has room for every head (more,
@@ -246,8 +259,27 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
     jobs[nj++] = PrepJob{PREP_PROJ, (const bf*)w_proj, (const bf*)b_proj, (unsigned char*)sc + fs.pimg[i],
                          (float*)(sc + fs.pbias[i]), p.C, p.d, p.dp, 0, 0, i * tp.NB, tp.NB, tp.natoms * 64, p.Ap,
                          fold_pbias ? 1 : 0};
-  int rc = launch_prep(jobs, nj, st);
-  if (rc) return rc;
+  int rc = GSWA_OK;
+  if (want_L) {
+    // images of the backward GEMMs (see BwdImages), in the same launch when the job table has room
+    Unit bunits[kMaxUnits];
+    const int bnu = make_units(p, bunits, 3);
+    TokenSplit tx;
+    if (bnu <= 0 || !token_split(p.C, 3 * p.Ap, &tx)) return GSWA_ERR_UNSUPPORTED;
+    const BwdImages bi = bwd_images(p, bunits, bnu, tx);
+    unsigned char* base = reinterpret_cast<unsigned char*>(sv + p.off_bimg);
+    if (nj + bnu + tx.nsplit > 16) {
+      if ((rc = launch_prep(jobs, nj, st))) return rc;
+      nj = 0;
+    }
+    for (int i = 0; i < bnu; ++i)
+      jobs[nj++] = PrepJob{PREP_PROJ_T, (const bf*)w_proj, nullptr, base + bi.img[i], nullptr, p.C, p.d,
+                           p.dp, bunits[i].h0, bunits[i].nheads, 0, bunits[i].nheads * p.dp, p.Cp, p.Ap};
+    for (int i = 0; i < tx.nsplit; ++i)
+      jobs[nj++] = PrepJob{PREP_QKV_T, (const bf*)w_qkv, nullptr, base + bi.ximg[i], nullptr, p.C, p.d,
+                           p.dp, 0, 0, i * tx.NB, tx.NB, tx.natoms * 64, p.Ap};
+  }
+  if ((rc = launch_prep(jobs, nj, st))) return rc;
 
   const float qscale = 1.4426950408889634f / sqrtf((float)p.d);   // d^-1/2 and log2(e): attention works in the log2 domain
   int maxh = 0;
@@ -322,7 +354,7 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
   const int nu = make_units(p, units, 3);
   TokenSplit tx;
   if (nu <= 0 || !token_split(p.C, 3 * p.Ap, &tx)) return GSWA_ERR_UNSUPPORTED;
-  const BwdScratch bs = bwd_layout(p, units, nu, tx);
+  const BwdScratch bs = bwd_layout(p);
   const FastGeom geo = make_geom(p);
   char* sc = static_cast<char*>(scratch);
   const char* sv = static_cast<const char*>(saved);
@@ -335,16 +367,9 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
   float* dummy = reinterpret_cast<float*>(sc + bs.dummy);
   if (cudaMemsetAsync(err, 0, 256, st) != cudaSuccess) return check_launch();
 
-  PrepJob jobs[16];
-  int nj = 0;
-  for (int i = 0; i < nu; ++i)
-    jobs[nj++] = PrepJob{PREP_PROJ_T, (const bf*)w_proj, nullptr, (unsigned char*)sc + bs.img[i], nullptr, p.C, p.d,
-                         p.dp, units[i].h0, units[i].nheads, 0, units[i].nheads * p.dp, p.Cp, p.Ap};
-  for (int i = 0; i < tx.nsplit; ++i)
-    jobs[nj++] = PrepJob{PREP_QKV_T, (const bf*)w_qkv, nullptr, (unsigned char*)sc + bs.ximg[i], nullptr, p.C, p.d,
-                         p.dp, 0, 0, i * tx.NB, tx.NB, tx.natoms * 64, p.Ap};
-  int rc = launch_prep(jobs, nj, st);
-  if (rc) return rc;
+  int rc = GSWA_OK;
+  const BwdImages bi = bwd_images(p, units, nu, tx);          // built by the forward call
+  const unsigned char* bimg = reinterpret_cast<const unsigned char*>(sv + p.off_bimg);
 
   if (dw_proj || db_proj) {
     // dW^P = dy^T A (A fetched by TMA); db^P rides on the ones column of A when the head dim is padded
@@ -369,7 +394,7 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
     GWUnit& w = gw.u[i];
     w.A = (const bf*)dy; w.lda = p.C; w.kvalid = p.C;
     w.H = p.H; w.W = p.W; w.s = p.gs[u.g]; w.nW = p.nW; w.nWw = p.nWw; w.n_windows = geo.n_windows;
-    w.Bimg = (const unsigned char*)sc + bs.img[i];
+    w.Bimg = bimg + bi.img[i];
     w.bias = nullptr;
     w.out = dO + geo.do_off[u.g] + (long long)(u.h0 - p.gh0[u.g]) * 64 * p.dp;
     w.win_stride = (long long)p.gh[u.g] * 64 * p.dp;
@@ -407,7 +432,7 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
     gt.out = (bf*)dx; gt.ldo = p.C; gt.NB = tx.NB; gt.nstages = tx.nstages; gt.stream_b = tx.stream_b; gt.err = err;
     for (int i = 0; i < tx.nsplit; ++i) {
       const int col0 = i * tx.NB;
-      gt.s[i] = GTSplit{(const unsigned char*)sc + bs.ximg[i], nullptr, col0, (p.C - col0 < tx.NB ? p.C - col0 : tx.NB)};
+      gt.s[i] = GTSplit{bimg + bi.ximg[i], nullptr, col0, (p.C - col0 < tx.NB ? p.C - col0 : tx.NB)};
     }
     if ((rc = launch_gt(gt, tx.nsplit, st, "dx_gemm"))) return rc;
   }

@@ -28,7 +28,7 @@ struct Plan {
   int Cp;                      // C padded to a multiple of 64 (K of the GEMMs that read the caller's rows)
   int Ap;                      // heads * dp: row length of the padded attention output
   // byte offsets inside `saved`
-  size_t off_qkv, off_A, off_L, saved_bytes;
+  size_t off_qkv, off_A, off_L, off_bimg, saved_bytes;   // off_bimg: weight images of the backward GEMMs (built by the forward call)
   size_t fwd_scratch, infer_scratch, bwd_scratch;
 };
 
