@@ -157,8 +157,9 @@ struct WinCtx {
 __device__ __forceinline__ WinCtx window_setup(const FastGeom& g, int s, long long win, int* tok, unsigned char* reg,
                                                int tid) {
   WinCtx c;
-  c.b = (int)(win / g.nW);
-  const int w = (int)(win % g.nW);
+  const int wn = (int)win;                       // window counts of this path fit 32 bits: no 64-bit division
+  c.b = wn / g.nW;
+  const int w = wn - c.b * g.nW;
   c.wi = w / g.nWw;
   c.wj = w % g.nWw;
   c.masked = s > 0 && (c.wi == g.nWh - 1 || c.wj == g.nWw - 1);
