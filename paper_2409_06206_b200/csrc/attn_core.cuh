@@ -157,17 +157,27 @@ struct WinCtx {
 __device__ __forceinline__ WinCtx window_setup(const FastGeom& g, int s, long long win, int* tok, unsigned char* reg,
                                                int tid) {
   WinCtx c;
-  const int wn = (int)win;                       // window counts of this path fit 32 bits: no 64-bit division
-  c.b = wn / g.nW;
-  const int w = wn - c.b * g.nW;
-  c.wi = w / g.nWw;
-  c.wj = w % g.nWw;
+  // window -> (image, window row, window column) without integer division: quotient from a float reciprocal,
+  // corrected by one step (window counts of this path stay far below 2^24)
+  const int wn = (int)win;
+  int b = (int)(((float)wn + 0.5f) * (1.0f / (float)g.nW));
+  int w = wn - b * g.nW;
+  if (w < 0) { --b; w += g.nW; } else if (w >= g.nW) { ++b; w -= g.nW; }
+  int wi = (int)(((float)w + 0.5f) * (1.0f / (float)g.nWw));
+  int wj = w - wi * g.nWw;
+  if (wj < 0) { --wi; wj += g.nWw; } else if (wj >= g.nWw) { ++wi; wj -= g.nWw; }
+  c.b = b;
+  c.wi = wi;
+  c.wj = wj;
   c.masked = s > 0 && (c.wi == g.nWh - 1 || c.wj == g.nWw - 1);
   if (tid < 64) {
-    int i, j, r;
-    slot_to_token(g.H, g.W, 8, s, w, tid, &i, &j, &r);
-    tok[tid] = (c.b * g.H + i) * g.W + j;
-    reg[tid] = (unsigned char)r;
+    // slot tid of the window in the shifted frame -> original token and mask label (what slot_to_token computes)
+    const int ip = wi * 8 + (tid >> 3), jp = wj * 8 + (tid & 7);
+    int i = ip + s, j = jp + s;
+    if (i >= g.H) i -= g.H;
+    if (j >= g.W) j -= g.W;
+    tok[tid] = (b * g.H + i) * g.W + j;
+    reg[tid] = (unsigned char)(3 * axis_region(ip, g.H, 8, s) + axis_region(jp, g.W, 8, s));
   }
   return c;
 }
