@@ -283,6 +283,7 @@ __global__ void __maxnreg__(96) attn_bwd_tc_kernel(const __grid_constant__ AttnL
 #pragma unroll
     for (int k = 0; k < 32; ++k) dsum[k] = 0.f;
     int pending = -1;                                      // input slot whose release waits for this thread's stores
+    const float inv_nW = 1.0f / (float)g.nW, inv_nWw = 1.0f / (float)g.nWw;
     // Staging layout of a window that wraps around the image edge: its four pieces (upper/lower rows x
     // left/right columns, split after 8 - s positions) one after the other, each in box order, unswizzled.
     const bool wrap_tma = u.s > 0 && u.s == L.wrap_s;
@@ -294,7 +295,11 @@ __global__ void __maxnreg__(96) attn_bwd_tc_kernel(const __grid_constant__ AttnL
       const int slot = i % kTcStages;
       const int win = 2 * (int)(first - (long long)i * gridDim.x) + x;
       const bool valid = win < (int)g.n_windows;
-      const int b = win / g.nW, wl = win - b * g.nW, wi = wl / g.nWw, wj = wl - wi * g.nWw;
+      // (image, window row, window column) without integer division: float reciprocal, corrected by one step
+      int b = (int)(((float)win + 0.5f) * inv_nW), wl = win - b * g.nW;
+      if (wl < 0) { --b; wl += g.nW; } else if (wl >= g.nW) { ++b; wl -= g.nW; }
+      int wi = (int)(((float)wl + 0.5f) * inv_nWw), wj = wl - wi * g.nWw;
+      if (wj < 0) { --wi; wj += g.nWw; } else if (wj >= g.nWw) { ++wi; wj -= g.nWw; }
       // A window in the last row or column of a shifted frame wraps around the image edge and carries mask
       // labels; along such an axis the first 8 - s positions have one label, the rest another.  Bit j of
       // `msk` = this query may attend to key 32 half + j.
