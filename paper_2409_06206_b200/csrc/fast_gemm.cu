@@ -1,11 +1,12 @@
 // Projection GEMMs of the bf16 path on the 5th-generation tensor cores (tcgen05.mma, accumulators in
 // TMEM).  Three persistent, warp-specialised kernels share one structure:
-//     warps 0-3  epilogue   TMEM -> registers -> global        (one accumulator row per thread)
-//     warp  4    MMA issue  one elected thread, tcgen05.mma + tcgen05.commit
-//     warps 5-12 loaders    global -> registers -> swizzled shared memory (row pitches of C = 60/180
-//                           elements are not 16-byte multiples, so the caller's tensors cannot be
-//                           described to TMA; rows are fetched with 8-byte loads and K is zero-padded
-//                           on the fly)
+//     epilogue warps   TMEM -> registers -> shared-memory staging -> global (one accumulator row per thread;
+//                      four in gr_kernel, eight in gw_kernel and gt_kernel: two per 32-lane TMEM quadrant)
+//     one MMA warp     one elected thread, tcgen05.mma + tcgen05.commit
+//     producers        padded token-major buffers (attention output, dqkv) come by TMA from one thread; the
+//                      caller's tensors (x, dy) have row pitches of 2C bytes (360 at C = 180), which cannot be
+//                      described to TMA: eight loader warps fetch their rows with asynchronous 8- and 16-byte
+//                      copies straight into the swizzled operand image, K padded on the fly
 // Roles talk through mbarriers; every wait is bounded and reports through an error word.
 //
 //   gw_kernel  Eq. 6 projections (and dA = dy W^P): rows are gathered in WINDOW order of one head
