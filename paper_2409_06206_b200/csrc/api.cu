@@ -39,6 +39,8 @@ KernelScope::~KernelScope() {
   if (slot < (int)g_prof.size()) cudaEventRecord(g_prof[slot].e1, st);
 }
 
+bool profiling_enabled() { return g_prof_on; }
+
 int check_launch() {
   const cudaError_t e = cudaGetLastError();
   if (e == cudaSuccess) return GSWA_OK;

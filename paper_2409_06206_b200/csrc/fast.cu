@@ -7,6 +7,8 @@
 
 #include "fast.cuh"
 
+#include <mutex>
+
 namespace gswa {
 namespace {
 
@@ -201,6 +203,33 @@ void fast_plan_sizes(Plan* p) {
   p->bwd_scratch = bwd_layout(*p).total;
 }
 
+// A second stream per device for the two weight-gradient GEMMs of the backward pass.  Nothing downstream reads
+// dW_proj or dW_qkv, so these kernels need not sit on the critical path: forked off the caller's stream with
+// events, their ramp-down (every CTA adding its accumulator into the gradients through the L2 atomic units, SMs
+// mostly idle) overlaps the start of the next kernel, whose CTAs take over the SMs as they come free.
+struct SideStream {
+  cudaStream_t s;
+  cudaEvent_t fork1, fork2, join;
+};
+static SideStream* side_stream() {
+  static std::mutex mu;
+  static SideStream table[64];
+  static int state[64];                     // 0 not tried, 1 ready, -1 unavailable
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { (void)cudaGetLastError(); return nullptr; }
+  std::lock_guard<std::mutex> lk(mu);
+  if (state[dev] == 0) {
+    SideStream& t = table[dev];
+    const bool ok = cudaStreamCreateWithFlags(&t.s, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&t.fork1, cudaEventDisableTiming) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&t.fork2, cudaEventDisableTiming) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&t.join, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) (void)cudaGetLastError();
+    state[dev] = ok ? 1 : -1;
+  }
+  return state[dev] == 1 ? &table[dev] : nullptr;
+}
+
 // Work units of the attention kernels: one head per CTA when the unit table has room for every head (more,
 // smaller CTAs per SM hide each other's latency), otherwise the head ranges of the GEMM units.
 static void attn_units(const Plan& p, const FastGeom& geo, const Unit* units, int nu, AttnLaunch* L) {
@@ -368,6 +397,10 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
   if (cudaMemsetAsync(err, 0, 256, st) != cudaSuccess) return check_launch();
 
   int rc = GSWA_OK;
+  // the weight-gradient GEMMs go to the side stream (not while kernels are being timed one by one)
+  SideStream* ss = profiling_enabled() ? nullptr : side_stream();
+  cudaStream_t s2 = ss ? ss->s : st;
+  if (ss && (cudaEventRecord(ss->fork1, st) != cudaSuccess || cudaStreamWaitEvent(s2, ss->fork1, 0) != cudaSuccess)) return check_launch();
   const BwdImages bi = bwd_images(p, units, nu, tx);          // built by the forward call
   const unsigned char* bimg = reinterpret_cast<const unsigned char*>(sv + p.off_bimg);
 
@@ -381,8 +414,8 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
     gr.Ap = p.Ap; gr.dp = p.dp; gr.d = p.d; gr.C = p.C; gr.M = gs.M; gr.rows = p.T;
     gr.NP = gs.NP; gr.mbpc = gs.mbpc; gr.nsplit = gs.nsplit;
     gr.out = dw_proj ? dw_proj : dummy; gr.colsum = p.d < p.dp ? db_proj : nullptr; gr.err = err;
-    if ((rc = launch_gr(gr, st, "dwproj_gemm"))) return rc;
-    if (db_proj && p.d == p.dp && (rc = launch_colsum_bf16((const bf*)dy, p.T, p.C, p.C, db_proj, st))) return rc;
+    if ((rc = launch_gr(gr, s2, "dwproj_gemm"))) return rc;
+    if (db_proj && p.d == p.dp && (rc = launch_colsum_bf16((const bf*)dy, p.T, p.C, p.C, db_proj, s2))) return rc;
   }
 
   // (dW^P runs first so that the dO tiles written next are still in L2 when the attention kernel reads them)
@@ -424,6 +457,8 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
     }
     if ((rc = launch_attn_bwd_tc(al, st))) return rc;
   } else if ((rc = launch_attn_bwd(al, st))) return rc;
+  // dqkv is complete on the caller's stream: dW_qkv may start on the side stream, next to dx
+  if (ss && (cudaEventRecord(ss->fork2, st) != cudaSuccess || cudaStreamWaitEvent(s2, ss->fork2, 0) != cudaSuccess)) return check_launch();
 
   if (dx) {
     GTLaunch gt{};
@@ -446,8 +481,10 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
     gr.Ap = p.Ap; gr.dp = p.dp; gr.d = p.d; gr.C = p.C; gr.M = gs.M; gr.rows = p.T;
     gr.NP = gs.NP; gr.mbpc = gs.mbpc; gr.nsplit = gs.nsplit;
     gr.out = dw_qkv ? dw_qkv : dummy; gr.colsum = db_qkv; gr.err = err;
-    if ((rc = launch_gr(gr, st, "dwqkv_gemm"))) return rc;
+    if ((rc = launch_gr(gr, s2, "dwqkv_gemm"))) return rc;
   }
+  // the caller's stream continues only after the side stream's work
+  if (ss && (cudaEventRecord(ss->join, s2) != cudaSuccess || cudaStreamWaitEvent(st, ss->join, 0) != cudaSuccess)) return check_launch();
   return GSWA_OK;
 }
 
