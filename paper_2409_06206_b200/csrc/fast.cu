@@ -210,6 +210,7 @@ void fast_plan_sizes(Plan* p) {
 struct SideStream {
   cudaStream_t s;
   cudaEvent_t fork1, fork2, join;
+  std::mutex use;               // one backward call at a time enqueues on it (its events are re-recorded per call)
 };
 static SideStream* side_stream() {
   static std::mutex mu;
@@ -399,6 +400,8 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
   int rc = GSWA_OK;
   // the weight-gradient GEMMs go to the side stream (not while kernels are being timed one by one)
   SideStream* ss = profiling_enabled() ? nullptr : side_stream();
+  std::unique_lock<std::mutex> ss_lock;
+  if (ss) ss_lock = std::unique_lock<std::mutex>(ss->use);
   cudaStream_t s2 = ss ? ss->s : st;
   if (ss && (cudaEventRecord(ss->fork1, st) != cudaSuccess || cudaStreamWaitEvent(s2, ss->fork1, 0) != cudaSuccess)) return check_launch();
   const BwdImages bi = bwd_images(p, units, nu, tx);          // built by the forward call
