@@ -203,11 +203,9 @@ int gswa_backward(const gswa_desc* desc, const void* x, const void* w_qkv, const
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (!(p.flags & GSWA_FLAG_ACCUMULATE)) {
     const size_t C = (size_t)p.C, nrel = (size_t)(2 * p.M - 1) * (2 * p.M - 1);
-    if (dw_qkv && (rc = cuda_rc(cudaMemsetAsync(dw_qkv, 0, 3 * C * C * sizeof(float), st)))) return rc;
-    if (db_qkv && (rc = cuda_rc(cudaMemsetAsync(db_qkv, 0, 3 * C * sizeof(float), st)))) return rc;
-    if (dw_proj && (rc = cuda_rc(cudaMemsetAsync(dw_proj, 0, C * C * sizeof(float), st)))) return rc;
-    if (db_proj && (rc = cuda_rc(cudaMemsetAsync(db_proj, 0, C * sizeof(float), st)))) return rc;
-    if (dbias_table && (rc = cuda_rc(cudaMemsetAsync(dbias_table, 0, nrel * p.nh * sizeof(float), st)))) return rc;
+    float* const ptrs[5] = {dw_qkv, db_qkv, dw_proj, db_proj, dbias_table};
+    const long long counts[5] = {(long long)(3 * C * C), (long long)(3 * C), (long long)(C * C), (long long)C, (long long)(nrel * p.nh)};
+    if ((rc = launch_zero(ptrs, counts, 5, st))) return rc;
   }
   if (p.T == 0) return GSWA_OK;
   if (p.fast)

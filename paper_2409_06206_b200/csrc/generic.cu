@@ -406,6 +406,27 @@ int generic_backward(const Plan& p, const void* x, const void* w_qkv, const void
                         (const bf*)dy, (bf*)dx, dw_qkv, db_qkv, dw_proj, db_proj, dtable, (char*)scratch, st);
 }
 
+// Zeroes up to six float buffers with one launch (the parameter gradients of a backward call: six separate
+// memsets cost six stream operations in front of the first kernel).
+struct ZeroJobs {
+  float* p[6];
+  long long n[6];
+};
+__global__ void zero_kernel(const __grid_constant__ ZeroJobs J) {
+  float* p = J.p[blockIdx.y];
+  const long long n = J.n[blockIdx.y];
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) p[i] = 0.f;
+}
+int launch_zero(float* const* ptrs, const long long* counts, int nbuf, cudaStream_t st) {
+  ZeroJobs J{};
+  int k = 0;
+  for (int i = 0; i < nbuf && k < 6; ++i)
+    if (ptrs[i] != nullptr && counts[i] > 0) { J.p[k] = ptrs[i]; J.n[k] = counts[i]; ++k; }
+  if (k == 0) return GSWA_OK;
+  { KernelScope ks_("zero_grads", st); zero_kernel<<<dim3(48, k), 256, 0, st>>>(J); }
+  return check_launch();
+}
+
 int launch_colsum_bf16(const __nv_bfloat16* G, long long rows, int cols, long long ld, float* out, cudaStream_t st) {
   return launch_colsum<__nv_bfloat16>(G, rows, cols, ld, out, st);
 }

@@ -39,6 +39,7 @@ struct HeadShifts {
 
 int make_plan(const gswa_desc* desc, Plan* plan);
 int check_launch();  // GSWA_OK or GSWA_ERR_CUDA (records the CUDA error text)
+int launch_zero(float* const* ptrs, const long long* counts, int nbuf, cudaStream_t st);   // one launch zeroes them all
 bool profiling_enabled();  // per-kernel event timing is on (kernels are then kept on one stream)
 
 // Wraps one kernel launch: counts it and, while profiling is enabled, brackets it with a CUDA
