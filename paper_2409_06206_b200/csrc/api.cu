@@ -201,11 +201,16 @@ int gswa_backward(const gswa_desc* desc, const void* x, const void* w_qkv, const
     return GSWA_ERR_ALIGN;
   if (scratch_bytes < p.bwd_scratch) return GSWA_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  if (!(p.flags & GSWA_FLAG_ACCUMULATE)) {
+  {
+    // one launch zeroes the parameter gradients (unless they accumulate) and, on the tensor-core path, the error
+    // word at the head of the scratch buffer
     const size_t C = (size_t)p.C, nrel = (size_t)(2 * p.M - 1) * (2 * p.M - 1);
-    float* const ptrs[5] = {dw_qkv, db_qkv, dw_proj, db_proj, dbias_table};
-    const long long counts[5] = {(long long)(3 * C * C), (long long)(3 * C), (long long)(C * C), (long long)C, (long long)(nrel * p.nh)};
-    if ((rc = launch_zero(ptrs, counts, 5, st))) return rc;
+    const bool z = !(p.flags & GSWA_FLAG_ACCUMULATE);
+    float* const ptrs[6] = {z ? dw_qkv : nullptr, z ? db_qkv : nullptr, z ? dw_proj : nullptr, z ? db_proj : nullptr,
+                            z ? dbias_table : nullptr, p.fast && p.T > 0 ? static_cast<float*>(scratch) : nullptr};
+    const long long counts[6] = {(long long)(3 * C * C), (long long)(3 * C), (long long)(C * C), (long long)C,
+                                 (long long)(nrel * p.nh), 64};
+    if ((rc = launch_zero(ptrs, counts, 6, st))) return rc;
   }
   if (p.T == 0) return GSWA_OK;
   if (p.fast)

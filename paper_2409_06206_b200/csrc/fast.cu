@@ -273,7 +273,6 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
   bf* qkv = reinterpret_cast<bf*>(sv + p.off_qkv);
   bf* A = reinterpret_cast<bf*>(sv + p.off_A);
   float* Lt = reinterpret_cast<float*>(sv + p.off_L);
-  if (cudaMemsetAsync(err, 0, 256, st) != cudaSuccess) return check_launch();
 
   // With a spare K column (C < Cp) the QKV bias rides in the weight image and meets a column of ones in the A operand.
   const bool fold_bias = p.C < p.Cp && b_qkv != nullptr && !(p.flags & GSWA_FLAG_FUSED_FWD);
@@ -299,7 +298,7 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
     const BwdImages bi = bwd_images(p, bunits, bnu, tx);
     unsigned char* base = reinterpret_cast<unsigned char*>(sv + p.off_bimg);
     if (nj + bnu + tx.nsplit > 16) {
-      if ((rc = launch_prep(jobs, nj, st))) return rc;
+      if ((rc = launch_prep(jobs, nj, st, err))) return rc;
       nj = 0;
     }
     for (int i = 0; i < bnu; ++i)
@@ -309,7 +308,7 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
       jobs[nj++] = PrepJob{PREP_QKV_T, (const bf*)w_qkv, nullptr, base + bi.ximg[i], nullptr, p.C, p.d,
                            p.dp, 0, 0, i * tx.NB, tx.NB, tx.natoms * 64, p.Ap};
   }
-  if ((rc = launch_prep(jobs, nj, st))) return rc;
+  if ((rc = launch_prep(jobs, nj, st, err))) return rc;     // also zeroes the error word
 
   const float qscale = 1.4426950408889634f / sqrtf((float)p.d);   // d^-1/2 and log2(e): attention works in the log2 domain
   int maxh = 0;
@@ -394,8 +393,7 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
   const float* Lt = reinterpret_cast<const float*>(sv + p.off_L);
   bf* dO = reinterpret_cast<bf*>(sc + bs.dO);
   bf* dqkv = reinterpret_cast<bf*>(sc + bs.dqkv);
-  float* dummy = reinterpret_cast<float*>(sc + bs.dummy);
-  if (cudaMemsetAsync(err, 0, 256, st) != cudaSuccess) return check_launch();
+  float* dummy = reinterpret_cast<float*>(sc + bs.dummy);      // (the error word was zeroed together with the gradients)
 
   int rc = GSWA_OK;
   // the weight-gradient GEMMs go to the side stream (not while kernels are being timed one by one)

@@ -163,7 +163,7 @@ struct PrepJob {
   int Ap;                      // heads * dp: K of PREP_PROJ / PREP_QKV_T runs over padded (kind, head, c) indices
   int fold_bias;               // PREP_QKV: write the bias into image row k == C (needs C < KP) instead of bias_out
 };
-int launch_prep(const PrepJob* jobs, int njobs, cudaStream_t st);
+int launch_prep(const PrepJob* jobs, int njobs, cudaStream_t st, int* err_word = nullptr);   // err_word: 64 ints zeroed by the same launch
 
 // ---- attention (mma.sync m16n8k16, softmax in registers)
 struct AttnUnit {

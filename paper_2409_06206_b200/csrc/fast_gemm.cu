@@ -681,6 +681,7 @@ __global__ void __launch_bounds__(kThreadsR, 1) gr_kernel(const __grid_constant_
 // ==========================================================================================
 struct PrepJobs {
   PrepJob j[16];
+  int* err_word;               // or nullptr: 64 ints zeroed by block (0, 0)
 };
 
 // Value of image element (row n, K index k) and of the bias that goes with row n.
@@ -708,6 +709,7 @@ __device__ __forceinline__ float prep_value(const PrepJob& p, int n, int k, int 
 // transposed ones), blocks along the other; the padded head width is a power of two, so nothing divides per element.
 __global__ void __launch_bounds__(256) prep_kernel(const __grid_constant__ PrepJobs J) {
   const PrepJob& p = J.j[blockIdx.y];
+  if (J.err_word != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 64) J.err_word[threadIdx.x] = 0;
   const int ldp = p.dp == 32 ? 5 : 4, dmask = p.dp - 1;
   const bool transposed = p.mode == PREP_PROJ_T || p.mode == PREP_QKV_T;
   const int nouter = transposed ? p.KP : p.NT, ninner = transposed ? p.NT : p.KP;
@@ -734,11 +736,12 @@ __global__ void __launch_bounds__(256) prep_kernel(const __grid_constant__ PrepJ
 
 }  // namespace
 
-int launch_prep(const PrepJob* jobs, int njobs, cudaStream_t st) {
+int launch_prep(const PrepJob* jobs, int njobs, cudaStream_t st, int* err_word) {
   if (njobs <= 0) return GSWA_OK;
   if (njobs > 16) return GSWA_ERR_UNSUPPORTED;
   PrepJobs J{};
   for (int i = 0; i < njobs; ++i) J.j[i] = jobs[i];
+  J.err_word = err_word;
   { KernelScope ks_("prep_weights", st); prep_kernel<<<dim3(96, njobs), 256, 0, st>>>(J); }
   return check_launch();
 }
