@@ -524,7 +524,7 @@ __global__ void __launch_bounds__(kThreadsR, 1) gr_kernel(const __grid_constant_
       RingPos rp;
       rp.init(0, ST);
       for (int s = 0; s < nst; ++s) {
-        if (!wait_bar(&emptyT[rp.slot], rp.ph ^ 1, &abort_s, L.err)) break;
+        if (!wait_bar_nap(&emptyT[rp.slot], rp.ph ^ 1, &abort_s, L.err)) break;
         const uint32_t dst = smem_u32(ringT + (size_t)rp.slot * tbytes);
         mbar_arrive_expect_tx(&fullT[rp.slot], (uint32_t)tma_atoms * 8192u);
         for (int a = 0; a < tma_atoms; ++a)
@@ -556,7 +556,7 @@ __global__ void __launch_bounds__(kThreadsR, 1) gr_kernel(const __grid_constant_
     const uint32_t sS = smem_u32(base);
     int ph = 0;
     for (int s = set; s < nst; s += kSets, ph ^= 1) {
-      if (!wait_bar_warp(&emptyC[set], ph ^ 1, &abort_s, L.err)) break;
+      if (!wait_bar_warp_nap(&emptyC[set], ph ^ 1, &abort_s, L.err)) break;
       const long long tb = t0 + (long long)s * 64;
       const char* pp = srcP + (tb + ll.lw) * prow + (copy_col0 + ll.pp * 8) * 2;
       const bool whole = tb + 64 <= t1;
@@ -590,7 +590,7 @@ __global__ void __launch_bounds__(kThreadsR, 1) gr_kernel(const __grid_constant_
       bool ok = true;
       for (int s = 0; s < nst; ++s) {
         const int sc = s & (kSets - 1), pc = (s / kSets) & 1;
-        if (!wait_bar(&fullT[rt.slot], rt.ph, &abort_s, L.err) || !wait_bar(&fullC[sc], pc, &abort_s, L.err)) { ok = false; break; }
+        if (!wait_bar_nap(&fullT[rt.slot], rt.ph, &abort_s, L.err) || !wait_bar_nap(&fullC[sc], pc, &abort_s, L.err)) { ok = false; break; }
         fence_after_sync();
         const uint32_t tAddr = smem_u32(ringT + (size_t)rt.slot * tbytes), cAddr = smem_u32(ringC + (size_t)sc * cbytes);
         const uint32_t lAddr = L.tma_is_L ? tAddr : cAddr, rAddr = L.tma_is_L ? cAddr : tAddr;
@@ -618,7 +618,7 @@ __global__ void __launch_bounds__(kThreadsR, 1) gr_kernel(const __grid_constant_
         colmap[ni] = ni == ones ? -2 : (L.tma_is_L ? (ni < L.C ? ni : -1) : (ni < L.Ap ? unpad_index(ni, L.Ap, L.dp, L.d, L.C) : -1));
       asm volatile("bar.sync 1, 128;" ::: "memory");
     }
-    if (wait_bar_warp(&done, 0, &abort_s, L.err)) {
+    if (wait_bar_warp_nap(&done, 0, &abort_s, L.err)) {
       fence_after_sync();
       {
         // Atomic accumulation into the caller's gradients.  The padded row and column indices were turned into
