@@ -66,10 +66,12 @@ __device__ __forceinline__ void load_tiles(unsigned char* dst, const __nv_bfloat
 }
 
 // S (16 rows x 64 keys) = Q K^T for the warp's rows; returns accumulators in s[8][4].
-template <int DP>
+template <int DP, bool kZero = true>
 __device__ __forceinline__ void qk_scores(float (*s)[4], uint32_t q_base, uint32_t k_base, int r0, int lane) {
+  if constexpr (kZero) {
 #pragma unroll
-  for (int j = 0; j < 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+    for (int j = 0; j < 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+  }
 #pragma unroll
   for (int kk = 0; kk < DP / 16; ++kk) {
     uint32_t a[4];
@@ -182,19 +184,21 @@ __device__ __forceinline__ WinCtx window_setup(const FastGeom& g, int s, long lo
   return c;
 }
 
-// Adds the relative-position bias and applies the mask (scores are in the log2 domain throughout).
-__device__ __forceinline__ void bias_and_mask(float (*s)[4], const float* tab, const unsigned char* reg, bool masked,
-                                              int p0, int t) {
+// The scores start from the relative-position bias (the MMAs then accumulate q k^T on top of it: no separate
+// addition); q and the table are already scaled by log2(e), the scores are in the log2 domain throughout.
+__device__ __forceinline__ void bias_init(float (*s)[4], const float* tab, int p0, int t) {
   const int pa0 = p0 >> 3, pc0 = p0 & 7;   // rows p0 and p0 + 8: same column in the window, next row
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const int pa = pa0 + (e >> 1), qc = 2 * t + (e & 1);
-      const int rel = (pa - j + 7) * 15 + (pc0 - qc + 7);
-      s[j][e] += tab[rel];                  // q and the table are already scaled by log2(e)
+      s[j][e] = tab[(pa - j + 7) * 15 + (pc0 - qc + 7)];
     }
   }
+}
+// Window mask: pairs whose slots carry different region labels are excluded.
+__device__ __forceinline__ void apply_mask(float (*s)[4], const unsigned char* reg, bool masked, int p0, int t) {
   if (masked) {
     const unsigned char r0 = reg[p0], r1 = reg[p0 + 8];
 #pragma unroll
@@ -220,8 +224,9 @@ __device__ __forceinline__ void fwd_window(uint32_t q_base, uint32_t k_base, uin
                                            unsigned char* ostg, __nv_bfloat16* A, int Ap, int h, int d, float* lt) {
   const int gq = lane >> 2, t = lane & 3, p0 = r0 + gq;
   float s[8][4];
-  qk_scores<DP>(s, q_base, k_base, r0, lane);
-  bias_and_mask(s, tab, reg, masked, p0, t);
+  bias_init(s, tab, p0, t);
+  qk_scores<DP, false>(s, q_base, k_base, r0, lane);
+  apply_mask(s, reg, masked, p0, t);
 
   float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll

@@ -162,8 +162,9 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 4 : 1) attn_bwd_kernel(c
 
     // ---- query-major phase: this warp owns query rows r0 .. r0+15 of head hl
     float s[8][4];
-    qk_scores<DP>(s, q_base, k_base, r0, lane);
-    bias_and_mask(s, tab + hl * 225, reg, wc.masked, p0, t);
+    bias_init(s, tab + hl * 225, p0, t);
+    qk_scores<DP, false>(s, q_base, k_base, r0, lane);
+    apply_mask(s, reg, wc.masked, p0, t);
     const float l0 = Lrow[hl * 64 + p0] * kLog2e, l1 = Lrow[hl * 64 + p0 + 8] * kLog2e;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
