@@ -45,6 +45,41 @@ __device__ __forceinline__ float ex2(float x) {          // 2^x, one MUFU instru
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Two fp32 lanes per instruction (packed f32x2 arithmetic) and the three-input maximum: the softmax
+// arithmetic of these kernels is bound by instruction issue, and each of these halves an instruction count.
+__device__ __forceinline__ unsigned long long pk2(float a, float b) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void upk2(unsigned long long r, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(r));
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+  unsigned long long r;
+  asm("add.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ unsigned long long sub2(unsigned long long a, unsigned long long b) {
+  unsigned long long r;
+  asm("sub.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ unsigned long long mul2(unsigned long long a, unsigned long long b) {
+  unsigned long long r;
+  asm("mul.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 __device__ __forceinline__ void stsm_x4(uint32_t addr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3) {
   asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
                : "memory");
@@ -231,22 +266,33 @@ __device__ __forceinline__ void fwd_window(uint32_t q_base, uint32_t k_base, uin
   float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    m0 = fmaxf(m0, fmaxf(s[j][0], s[j][1]));
-    m1 = fmaxf(m1, fmaxf(s[j][2], s[j][3]));
+    m0 = max3(m0, s[j][0], s[j][1]);
+    m1 = max3(m1, s[j][2], s[j][3]);
   }
   m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1));
   m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
   m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1));
   m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
-  float sum0 = 0.f, sum1 = 0.f;
+  float sum0, sum1;
+  {
+    const unsigned long long mm0 = pk2(m0, m0), mm1 = pk2(m1, m1);
+    unsigned long long acc0 = pk2(0.f, 0.f), acc1 = acc0;
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    s[j][0] = ex2(s[j][0] - m0);
-    s[j][1] = ex2(s[j][1] - m0);
-    s[j][2] = ex2(s[j][2] - m1);
-    s[j][3] = ex2(s[j][3] - m1);
-    sum0 += s[j][0] + s[j][1];
-    sum1 += s[j][2] + s[j][3];
+    for (int j = 0; j < 8; ++j) {
+      upk2(sub2(pk2(s[j][0], s[j][1]), mm0), s[j][0], s[j][1]);
+      upk2(sub2(pk2(s[j][2], s[j][3]), mm1), s[j][2], s[j][3]);
+      s[j][0] = ex2(s[j][0]);
+      s[j][1] = ex2(s[j][1]);
+      s[j][2] = ex2(s[j][2]);
+      s[j][3] = ex2(s[j][3]);
+      acc0 = add2(acc0, pk2(s[j][0], s[j][1]));
+      acc1 = add2(acc1, pk2(s[j][2], s[j][3]));
+    }
+    float a, b;
+    upk2(acc0, a, b);
+    sum0 = a + b;
+    upk2(acc1, a, b);
+    sum1 = a + b;
   }
   sum0 += __shfl_xor_sync(0xffffffffu, sum0, 1);
   sum0 += __shfl_xor_sync(0xffffffffu, sum0, 2);

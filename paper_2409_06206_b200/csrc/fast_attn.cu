@@ -166,35 +166,49 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 4 : 1) attn_bwd_kernel(c
     qk_scores<DP, false>(s, q_base, k_base, r0, lane);
     apply_mask(s, reg, wc.masked, p0, t);
     const float l0 = Lrow[hl * 64 + p0] * kLog2e, l1 = Lrow[hl * 64 + p0 + 8] * kLog2e;
+    {
+      const unsigned long long ll0 = pk2(l0, l0), ll1 = pk2(l1, l1);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      s[j][0] = ex2(s[j][0] - l0);
-      s[j][1] = ex2(s[j][1] - l0);
-      s[j][2] = ex2(s[j][2] - l1);
-      s[j][3] = ex2(s[j][3] - l1);
+      for (int j = 0; j < 8; ++j) {
+        upk2(sub2(pk2(s[j][0], s[j][1]), ll0), s[j][0], s[j][1]);
+        upk2(sub2(pk2(s[j][2], s[j][3]), ll1), s[j][2], s[j][3]);
+        s[j][0] = ex2(s[j][0]);
+        s[j][1] = ex2(s[j][1]);
+        s[j][2] = ex2(s[j][2]);
+        s[j][3] = ex2(s[j][3]);
+      }
     }
     float dp[8][4];
     qk_scores<DP>(dp, do_base, v_base, r0, lane);          // dP = dO V^T
-    float d0 = 0.f, d1 = 0.f;
+    float d0, d1;
+    {
+      unsigned long long a0 = pk2(0.f, 0.f), a1 = a0;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      d0 += s[j][0] * dp[j][0] + s[j][1] * dp[j][1];
-      d1 += s[j][2] * dp[j][2] + s[j][3] * dp[j][3];
+      for (int j = 0; j < 8; ++j) {
+        a0 = fma2(pk2(s[j][0], s[j][1]), pk2(dp[j][0], dp[j][1]), a0);
+        a1 = fma2(pk2(s[j][2], s[j][3]), pk2(dp[j][2], dp[j][3]), a1);
+      }
+      float a, b;
+      upk2(a0, a, b);
+      d0 = a + b;
+      upk2(a1, a, b);
+      d1 = a + b;
     }
     d0 += __shfl_xor_sync(0xffffffffu, d0, 1);
     d0 += __shfl_xor_sync(0xffffffffu, d0, 2);
     d1 += __shfl_xor_sync(0xffffffffu, d1, 1);
     d1 += __shfl_xor_sync(0xffffffffu, d1, 2);
+    {
+      const unsigned long long dd0 = pk2(d0, d0), dd1 = pk2(d1, d1);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      dp[j][0] = s[j][0] * (dp[j][0] - d0);
-      dp[j][1] = s[j][1] * (dp[j][1] - d0);
-      dp[j][2] = s[j][2] * (dp[j][2] - d1);
-      dp[j][3] = s[j][3] * (dp[j][3] - d1);
-      dsum[j][0] += dp[j][0];
-      dsum[j][1] += dp[j][1];
-      dsum[j][2] += dp[j][2];
-      dsum[j][3] += dp[j][3];
+      for (int j = 0; j < 8; ++j) {
+        const unsigned long long e0 = mul2(pk2(s[j][0], s[j][1]), sub2(pk2(dp[j][0], dp[j][1]), dd0));
+        const unsigned long long e1 = mul2(pk2(s[j][2], s[j][3]), sub2(pk2(dp[j][2], dp[j][3]), dd1));
+        upk2(e0, dp[j][0], dp[j][1]);
+        upk2(e1, dp[j][2], dp[j][3]);
+        upk2(add2(pk2(dsum[j][0], dsum[j][1]), e0), dsum[j][0], dsum[j][1]);
+        upk2(add2(pk2(dsum[j][2], dsum[j][3]), e1), dsum[j][2], dsum[j][3]);
+      }
     }
     {
       // P and dS cross to the key-major phase through shared memory: four 8x8 blocks per stmatrix
