@@ -221,15 +221,22 @@ __device__ __forceinline__ WinCtx window_setup(const FastGeom& g, int s, long lo
 
 // The scores start from the relative-position bias (the MMAs then accumulate q k^T on top of it: no separate
 // addition); q and the table are already scaled by log2(e), the scores are in the log2 domain throughout.
-__device__ __forceinline__ void bias_init(float (*s)[4], const float* tab, int p0, int t) {
+__device__ __forceinline__ void bias_init(float (*s)[4], const float2* tab2, int p0, int t) {
   const int pa0 = p0 >> 3, pc0 = p0 & 7;   // rows p0 and p0 + 8: same column in the window, next row
+  // a thread's two columns of a key block are neighbours in the table: entry r of the pair table holds
+  // (table[r], table[r - 1]), so one 8-byte load fills two accumulators
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int pa = pa0 + (e >> 1), qc = 2 * t + (e & 1);
-      s[j][e] = tab[(pa - j + 7) * 15 + (pc0 - qc + 7)];
-    }
+    const int r = (pa0 - j + 7) * 15 + (pc0 - 2 * t + 7);
+    const float2 a = tab2[r], b = tab2[r + 15];
+    s[j][0] = a.x; s[j][1] = a.y; s[j][2] = b.x; s[j][3] = b.y;
+  }
+}
+// Fills the pair table of `nheads` heads from the bf16 table [225][nh] (scaled by log2(e)).
+__device__ __forceinline__ void fill_pair_table(float2* tab2, const __nv_bfloat16* table, int nh, int h0, int nheads, int tid, int nt) {
+  for (int e = tid; e < nheads * 225; e += nt) {
+    const int r = e % 225, hh = h0 + e / 225;
+    tab2[e] = make_float2(__bfloat162float(table[r * nh + hh]) * kLog2e, r > 0 ? __bfloat162float(table[(r - 1) * nh + hh]) * kLog2e : 0.f);
   }
 }
 // Window mask: pairs whose slots carry different region labels are excluded.
@@ -254,7 +261,7 @@ __device__ __forceinline__ void apply_mask(float (*s)[4], const unsigned char* r
 // rows through the warp's staging block `ostg` to `A` (padded token-major, row length Ap) and, if
 // `lt` is not null, the natural-log row log-sum-exp to lt[0..63] (this head's block of the L tile).
 template <int DP>
-__device__ __forceinline__ void fwd_window(uint32_t q_base, uint32_t k_base, uint32_t v_base, const float* tab,
+__device__ __forceinline__ void fwd_window(uint32_t q_base, uint32_t k_base, uint32_t v_base, const float2* tab,
                                            const int* tok, const unsigned char* reg, bool masked, int r0, int lane,
                                            unsigned char* ostg, __nv_bfloat16* A, int Ap, int h, int d, float* lt) {
   const int gq = lane >> 2, t = lane & 3, p0 = r0 + gq;
@@ -309,7 +316,8 @@ __device__ __forceinline__ void fwd_window(uint32_t q_base, uint32_t k_base, uin
   const float inv0 = 1.f / sum0, inv1 = 1.f / sum1;
 #pragma unroll
   for (int jn = 0; jn < DP / 8; ++jn) {
-    o[jn][0] *= inv0; o[jn][1] *= inv0; o[jn][2] *= inv1; o[jn][3] *= inv1;
+    upk2(mul2(pk2(o[jn][0], o[jn][1]), pk2(inv0, inv0)), o[jn][0], o[jn][1]);
+    upk2(mul2(pk2(o[jn][2], o[jn][3]), pk2(inv1, inv1)), o[jn][2], o[jn][3]);
   }
   store_tile<DP>(ostg, o, 1.f, reinterpret_cast<unsigned char*>(A + (long long)tok[p0] * Ap + h * DP),
                  reinterpret_cast<unsigned char*>(A + (long long)tok[p0 + 8] * Ap + h * DP), lane,

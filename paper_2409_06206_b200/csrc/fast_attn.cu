@@ -31,11 +31,11 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 7 : 2) attn_fwd_kernel(c
   extern __shared__ __align__(128) unsigned char sm[];
   const int nh_u = u.nheads;
   const int tile_bytes = nh_u * 3 * 64 * DP * 2;
-  float* tab = reinterpret_cast<float*>(sm + 2 * (size_t)tile_bytes);
+  float2* tab = reinterpret_cast<float2*>(sm + 2 * (size_t)tile_bytes);     // pair table, see bias_init
   int* tok2 = reinterpret_cast<int*>(tab + nh_u * 225);
   unsigned char* reg2 = reinterpret_cast<unsigned char*>(tok2 + 128);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  unsigned char* ostg = sm + 2 * (size_t)tile_bytes + (((size_t)nh_u * 225 * 4 + 128 * 4 + 128 + 15) & ~(size_t)15) +
+  unsigned char* ostg = sm + 2 * (size_t)tile_bytes + (((size_t)nh_u * 225 * 8 + 128 * 4 + 128 + 15) & ~(size_t)15) +
                         (size_t)warp * 16 * DP * 2;                 // this warp's 16 x DP output staging block
   const int nt = nh_u * 128;
   __shared__ uint64_t ldbar[2];
@@ -47,8 +47,7 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 7 : 2) attn_fwd_kernel(c
   __syncthreads();
   if (tid >= nt) return;
 
-  for (int e = tid; e < nh_u * 225; e += nt)
-    tab[e] = __bfloat162float(L.table[(e % 225) * g.nh + u.h0 + e / 225]) * kLog2e;
+  fill_pair_table(tab, L.table, g.nh, u.h0, nh_u, tid, nt);
   const int hl = warp >> 2, r0 = (warp & 3) * 16;
   const int h = u.h0 + hl;
 
@@ -97,9 +96,9 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 4 : 1) attn_bwd_kernel(c
   unsigned char* Ps = sm + 2 * (size_t)in_bytes;               // [head][64][64] bf16
   unsigned char* dSs = Ps + (size_t)nh_u * 8192;
   float* Lrow2 = reinterpret_cast<float*>(dSs + (size_t)nh_u * 8192);   // [2][head][64], 16-byte aligned
-  float* tab = Lrow2 + 2 * nh_u * 64;
-  float* hist = tab + nh_u * 225;
-  int* tok2 = reinterpret_cast<int*>(hist + nh_u * 225);       // [2][64]
+  float2* tab = reinterpret_cast<float2*>(Lrow2 + 2 * nh_u * 64);          // pair table, see bias_init
+  float* hist = reinterpret_cast<float*>(sm);                  // per-offset sums of dS: built after the last window, over the dead input tiles
+  int* tok2 = reinterpret_cast<int*>(tab + nh_u * 225);        // [2][64]
   unsigned char* reg2 = reinterpret_cast<unsigned char*>(tok2 + 128);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   unsigned char* ostg = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(reg2 + 128) + 15) & ~(uintptr_t)15) +
@@ -114,10 +113,7 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 4 : 1) attn_bwd_kernel(c
   __syncthreads();
   if (tid >= nt) return;
 
-  for (int e = tid; e < nh_u * 225; e += nt) {
-    tab[e] = __bfloat162float(L.table[(e % 225) * g.nh + u.h0 + e / 225]) * kLog2e;
-    hist[e] = 0.f;
-  }
+  fill_pair_table(tab, L.table, g.nh, u.h0, nh_u, tid, nt);
   const int hl = warp >> 2, r0 = (warp & 3) * 16, gq = lane >> 2, t = lane & 3;
   const int h = u.h0 + hl;
   const int Ap = g.nh * DP;                                    // row length of the padded token-major buffers
@@ -267,6 +263,9 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 4 : 1) attn_bwd_kernel(c
 
   // ---- gradient of the bias table: fold this CTA's summed dS through the relative-position map
   if (L.dtable != nullptr) {
+    __syncthreads();                        // every warp has left the last window: its input tiles are dead
+    for (int e = tid; e < nh_u * 225; e += nt) hist[e] = 0.f;
+    __syncthreads();
     const int pa0 = p0 >> 3, pc0 = p0 & 7;
 #pragma unroll
     for (int j = 0; j < 8; ++j)
@@ -282,7 +281,7 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 4 : 1) attn_bwd_kernel(c
 
 template <int DP>
 size_t fwd_smem(int nheads) {
-  return (size_t)2 * nheads * 3 * 64 * DP * 2 + (size_t)nheads * 225 * 4 + 128 * 4 + 128 + 128 + (size_t)nheads * 4 * 16 * DP * 2;
+  return (size_t)2 * nheads * 3 * 64 * DP * 2 + (size_t)nheads * 225 * 8 + 128 * 4 + 128 + 128 + (size_t)nheads * 4 * 16 * DP * 2;
 }
 template <int DP>
 size_t bwd_smem(int nheads) {

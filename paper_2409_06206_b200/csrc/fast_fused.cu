@@ -47,7 +47,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) fw_kernel(const __grid_constant_
   unsigned char* ring = sB + (size_t)NT * CP * 2;
   unsigned char* tiles = ring + (size_t)S * kAtomBytes;          // q,k,v of one window: [head][kind][64][DP]
   float* sBias = reinterpret_cast<float*>(tiles + (size_t)nh_u * 3 * kTile);
-  float* tab = sBias + NT;
+  float2* tab = reinterpret_cast<float2*>(sBias + NT);        // pair table, see bias_init
   int* tok = reinterpret_cast<int*>(tab + nh_u * 225);
   unsigned char* reg = reinterpret_cast<unsigned char*>(tok + 64);
   unsigned char* ostg0 = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(reg + 64) + 15) & ~(uintptr_t)15);
@@ -59,8 +59,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) fw_kernel(const __grid_constant_
   for (int i = tid; i < NT * CP * 2 / 16; i += kThreadsF)
     reinterpret_cast<uint4*>(sB)[i] = __ldg(reinterpret_cast<const uint4*>(u.Bimg) + i);
   for (int i = tid; i < NT; i += kThreadsF) sBias[i] = u.bias ? u.bias[i] : 0.f;
-  for (int e = tid; e < nh_u * 225; e += kThreadsF)
-    tab[e] = __bfloat162float(L.table[(e % 225) * g.nh + u.h0 + e / 225]) * kLog2e;
+  attn::fill_pair_table(tab, L.table, g.nh, u.h0, nh_u, tid, kThreadsF);
   fence_proxy_async();
   if (tid == 0) {
     abort_s = 0;
@@ -270,7 +269,7 @@ int launch_fw_t(const FWLaunch& L, int nunits, cudaStream_t st) {
 size_t fw_smem_bytes(int Cp, int dp, int maxheads, int* nslots) {
   if (maxheads < 1 || maxheads > 3) return 0;
   const size_t NT = (size_t)maxheads * 3 * dp;
-  const size_t fixed = 1024 + NT * Cp * 2 + (size_t)maxheads * 3 * 64 * dp * 2 + NT * 4 + (size_t)maxheads * 225 * 4 + 64 * 4 + 64 +
+  const size_t fixed = 1024 + NT * Cp * 2 + (size_t)maxheads * 3 * 64 * dp * 2 + NT * 4 + (size_t)maxheads * 225 * 8 + 64 * 4 + 64 +
                        16 + (size_t)kAttnWarps * 16 * dp * 2 + 64;
   const size_t budget = 224 * 1024;
   const int need = Cp / 64 > kSetsF ? Cp / 64 : kSetsF;      // a tile's atoms must fit, and no more loader sets than slots
