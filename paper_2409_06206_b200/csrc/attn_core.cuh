@@ -150,17 +150,27 @@ __device__ __forceinline__ void set_word(uint4& v, int i, uint32_t w) {
 // token-major buffer: the tile is first laid out in the warp's 16 x DP staging block (stmatrix), then
 // every lane moves 16 bytes per row so that one store instruction covers whole 2*DP-byte row pieces.
 // `row0` / `row1` are the global addresses of the lane's two rows (fragment rows gq and gq + 8).
-template <int DP>
-__device__ __forceinline__ void store_tile(unsigned char* stg, const float (*acc)[4], float scale, unsigned char* row0,
-                                           unsigned char* row1, int lane, int ones_col) {
+// Fragment rows gq are multiplied by `scale0`, rows gq + 8 by `scale1` (kScaled = false: stored as they are).
+template <int DP, bool kScaled = true>
+__device__ __forceinline__ void store_tile(unsigned char* stg, const float (*acc)[4], float scale0, float scale1,
+                                           unsigned char* row0, unsigned char* row1, int lane, int ones_col) {
   const uint32_t sa = smem_u32(stg);
   const int m = lane >> 3;
+  const unsigned long long sc0 = pk2(scale0, scale0), sc1 = pk2(scale1, scale1);
 #pragma unroll
   for (int jn = 0; jn < DP / 8; jn += 2) {
     const int row = (m & 1) * 8 + (lane & 7), chunk = jn + (m >> 1);
-    stsm_x4(sa + tile_off<DP>(row, chunk), pack2(acc[jn][0] * scale, acc[jn][1] * scale),
-            pack2(acc[jn][2] * scale, acc[jn][3] * scale), pack2(acc[jn + 1][0] * scale, acc[jn + 1][1] * scale),
-            pack2(acc[jn + 1][2] * scale, acc[jn + 1][3] * scale));
+    float v[8];
+    if constexpr (kScaled) {
+      upk2(mul2(pk2(acc[jn][0], acc[jn][1]), sc0), v[0], v[1]);
+      upk2(mul2(pk2(acc[jn][2], acc[jn][3]), sc1), v[2], v[3]);
+      upk2(mul2(pk2(acc[jn + 1][0], acc[jn + 1][1]), sc0), v[4], v[5]);
+      upk2(mul2(pk2(acc[jn + 1][2], acc[jn + 1][3]), sc1), v[6], v[7]);
+    } else {
+      v[0] = acc[jn][0]; v[1] = acc[jn][1]; v[2] = acc[jn][2]; v[3] = acc[jn][3];
+      v[4] = acc[jn + 1][0]; v[5] = acc[jn + 1][1]; v[6] = acc[jn + 1][2]; v[7] = acc[jn + 1][3];
+    }
+    stsm_x4(sa + tile_off<DP>(row, chunk), pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
   }
   __syncwarp();
   if constexpr (DP == 32) {
@@ -314,12 +324,7 @@ __device__ __forceinline__ void fwd_window(uint32_t q_base, uint32_t k_base, uin
   // rows of the padded attention output: DP columns per head, pad columns are exact zeros because
   // the pad columns of v are; column d of head 0 is set to one (bias-gradient column, see fast.cuh)
   const float inv0 = 1.f / sum0, inv1 = 1.f / sum1;
-#pragma unroll
-  for (int jn = 0; jn < DP / 8; ++jn) {
-    upk2(mul2(pk2(o[jn][0], o[jn][1]), pk2(inv0, inv0)), o[jn][0], o[jn][1]);
-    upk2(mul2(pk2(o[jn][2], o[jn][3]), pk2(inv1, inv1)), o[jn][2], o[jn][3]);
-  }
-  store_tile<DP>(ostg, o, 1.f, reinterpret_cast<unsigned char*>(A + (long long)tok[p0] * Ap + h * DP),
+  store_tile<DP>(ostg, o, inv0, inv1, reinterpret_cast<unsigned char*>(A + (long long)tok[p0] * Ap + h * DP),
                  reinterpret_cast<unsigned char*>(A + (long long)tok[p0 + 8] * Ap + h * DP), lane,
                  (h == 0 && d < DP) ? d : -1);
   if (lt != nullptr && t == 0) {

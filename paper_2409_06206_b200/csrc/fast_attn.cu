@@ -226,7 +226,7 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 4 : 1) attn_bwd_kernel(c
 #pragma unroll
       for (int j = 0; j < DP / 8; ++j) dq[j][0] = dq[j][1] = dq[j][2] = dq[j][3] = 0.f;
       regs_times_tile<DP>(dq, dp, k_base, lane);             // dQ = dS K
-      store_tile<DP>(ostg, dq, L.scale, drow0, drow1, lane, -1);
+      store_tile<DP>(ostg, dq, L.scale, L.scale, drow0, drow1, lane, -1);
     }
     __syncthreads();
 
@@ -257,8 +257,8 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 4 : 1) attn_bwd_kernel(c
       }
     }
     // q was stored scaled by log2(e) (the scores live in the log2 domain): dK = dS^T q takes it back out
-    store_tile<DP>(ostg, dk, kLn2, drow0 + Ap * 2, drow1 + Ap * 2, lane, -1);
-    store_tile<DP>(ostg, dv, 1.f, drow0 + Ap * 4, drow1 + Ap * 4, lane, -1);
+    store_tile<DP>(ostg, dk, kLn2, kLn2, drow0 + Ap * 2, drow1 + Ap * 2, lane, -1);
+    store_tile<DP, false>(ostg, dv, 1.f, 1.f, drow0 + Ap * 4, drow1 + Ap * 4, lane, -1);
   }
 
   // ---- gradient of the bias table: fold this CTA's summed dS through the relative-position map
