@@ -426,7 +426,7 @@ def kernel_cost(cfg: LayerConfig, name: str):
 # DRAM bytes per token of each kernel, dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture
 # on workload c3 (131072 tokens; traffic grows in proportion to the tokens) divided by its tokens.
 # None = not captured since the kernel last changed.  Source: profiles/.
-NCU_DRAM_BYTES_PER_TOKEN = {"attn_bwd": 315.86e6 / 131072}   # profiles/attn_bwd_c3_ncu.md
+NCU_DRAM_BYTES_PER_TOKEN = {"attn_bwd": 314.09e6 / 131072}   # profiles/attn_bwd_c3_ncu.md
 
 
 def dominant_roofline(cfg, kernels, pk, pk_src):
