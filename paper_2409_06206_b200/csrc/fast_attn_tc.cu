@@ -279,9 +279,9 @@ __global__ void __maxnreg__(96) attn_bwd_tc_kernel(const __grid_constant__ AttnL
     float* dpart = Dx + (grp * 2 + (half ^ 1)) * 128 + r;      // where the partner reads this thread's part of D
     const float* dpeer = Dx + (grp * 2 + half) * 128 + r;
     const int pair_id = 1 + grp * 4 + wq, win_id = 9 + grp * 2 + x;
-    float dsum[32];
+    unsigned long long dsum2[16];                           // per-key sums of dS, two keys per packed f32x2 word
 #pragma unroll
-    for (int k = 0; k < 32; ++k) dsum[k] = 0.f;
+    for (int k = 0; k < 16; ++k) dsum2[k] = attn::pk2(0.f, 0.f);
     int pending = -1;                                      // input slot whose release waits for this thread's stores
     const float inv_nW = 1.0f / (float)g.nW, inv_nWw = 1.0f / (float)g.nWw;
     // Staging layout of a window that wraps around the image edge: its four pieces (upper/lower rows x
@@ -323,6 +323,8 @@ __global__ void __maxnreg__(96) attn_bwd_tc_kernel(const __grid_constant__ AttnL
       float D = 0.f;
       if (ok && valid) {
         const float l2 = Ls[slot * 128 + r] * kLog2e;
+        const unsigned long long l22 = attn::pk2(l2, l2);
+        unsigned long long D2 = attn::pk2(0.f, 0.f);
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
           uint32_t sv[16], dv[16], pk[8];
@@ -332,20 +334,29 @@ __global__ void __maxnreg__(96) attn_bwd_tc_kernel(const __grid_constant__ AttnL
 #pragma unroll
           for (int j = 0; j < 16; j += 2) {
             const int k0 = c * 16 + j, k1 = k0 + 1;
-            float p0 = ex2(__uint_as_float(sv[j]) + tabq[-(k0 >> 3) * kTabPitch - (k0 & 7)] - l2);
-            float p1 = ex2(__uint_as_float(sv[j + 1]) + tabq[-(k1 >> 3) * kTabPitch - (k1 & 7)] - l2);
+            float p0, p1;
+            attn::upk2(attn::sub2(attn::add2(attn::pk2(__uint_as_float(sv[j]), __uint_as_float(sv[j + 1])),
+                                             attn::pk2(tabq[-(k0 >> 3) * kTabPitch - (k0 & 7)], tabq[-(k1 >> 3) * kTabPitch - (k1 & 7)])),
+                                  l22),
+                       p0, p1);
+            p0 = ex2(p0);
+            p1 = ex2(p1);
             if (wmasked) {
               if (!((msk >> k0) & 1u)) p0 = 0.f;
               if (!((msk >> k1) & 1u)) p1 = 0.f;
             }
-            D = fmaf(p0, __uint_as_float(dv[j]), D);
-            D = fmaf(p1, __uint_as_float(dv[j + 1]), D);
+            D2 = attn::fma2(attn::pk2(p0, p1), attn::pk2(__uint_as_float(dv[j]), __uint_as_float(dv[j + 1])), D2);
             pk[j >> 1] = pack_bf16(p0, p1);
           }
           // P goes to its block at once (16 keys = two 16-byte chunks of the row, 128-byte swizzle); the second
           // pass reads it back, which keeps it out of the registers in between
           st_shared_v4(prow + (((uint32_t)(4 * half + 2 * c) ^ swz) << 4), pk[0], pk[1], pk[2], pk[3]);
           st_shared_v4(prow + (((uint32_t)(4 * half + 2 * c + 1) ^ swz) << 4), pk[4], pk[5], pk[6], pk[7]);
+        }
+        {
+          float da, db;
+          attn::upk2(D2, da, db);
+          D = da + db;
         }
         *dpart = D;
       }
@@ -357,6 +368,7 @@ __global__ void __maxnreg__(96) attn_bwd_tc_kernel(const __grid_constant__ AttnL
       ok = bar_vote(pair_id, 64, ok);                      // the two warps that share these rows
       if (ok && valid) {
         D += *dpeer;
+        const unsigned long long DD = attn::pk2(D, D);
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
           uint32_t dv[16], dsw[8], pk[8];
@@ -369,10 +381,11 @@ __global__ void __maxnreg__(96) attn_bwd_tc_kernel(const __grid_constant__ AttnL
           for (int j = 0; j < 16; j += 2) {
             const int k0 = c * 16 + j;
             const uint32_t w = pk[j >> 1];
-            const float ds0 = __uint_as_float(w << 16) * (__uint_as_float(dv[j]) - D);
-            const float ds1 = __uint_as_float(w & 0xFFFF0000u) * (__uint_as_float(dv[j + 1]) - D);
-            dsum[k0] += ds0;
-            dsum[k0 + 1] += ds1;
+            const unsigned long long ds2 = attn::mul2(attn::pk2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u)),
+                                                      attn::sub2(attn::pk2(__uint_as_float(dv[j]), __uint_as_float(dv[j + 1])), DD));
+            dsum2[k0 >> 1] = attn::add2(dsum2[k0 >> 1], ds2);
+            float ds0, ds1;
+            attn::upk2(ds2, ds0, ds1);
             dsw[j >> 1] = pack_bf16(ds0, ds1);
           }
           st_shared_v4(prow + 16384 + o0, dsw[0], dsw[1], dsw[2], dsw[3]);
@@ -465,7 +478,12 @@ __global__ void __maxnreg__(96) attn_bwd_tc_kernel(const __grid_constant__ AttnL
     // ---- gradient of the bias table: fold the summed dS of all rows through the relative-position map
     if (L.dtable != nullptr) {
 #pragma unroll
-      for (int k = 0; k < 32; ++k) atomicAdd(hist + (qa - 4 * half - (k >> 3) + 7) * 15 + (qc - (k & 7) + 7), dsum[k]);
+      for (int k = 0; k < 32; k += 2) {
+        float e0, e1;
+        attn::upk2(dsum2[k >> 1], e0, e1);
+        atomicAdd(hist + (qa - 4 * half - (k >> 3) + 7) * 15 + (qc - (k & 7) + 7), e0);
+        atomicAdd(hist + (qa - 4 * half - ((k + 1) >> 3) + 7) * 15 + (qc - ((k + 1) & 7) + 7), e1);
+      }
     }
     asm volatile("bar.sync 13, 512;" ::: "memory");        // all softmax warps
     if (L.dtable != nullptr && tid < 225) atomicAdd(L.dtable + tid * g.nh + u.h0, hist[tid]);
