@@ -98,7 +98,7 @@ def run_reference(args, cfg):
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": "tokens/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": workload_config(cfg),
+            "config": dict(workload_config(cfg), flags=args.flags),
             "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -232,6 +232,31 @@ def unfused_peak_bytes(cfg: LayerConfig, dev, batch: int):
 
 
 # ------------------------------------------------------------------------------ our arm
+def timed_repeats(args, step, barrier, check_status, gb):
+    """Times `--steps` steps, bracketed by a barrier and a device synchronisation on both sides, with CUDA events on
+    the launching stream, `--repeats` times over; the reported step time is the median repeat (max over ranks of
+    each).  After every repeat the device error word is read: a kernel that gave up a bounded wait returns early,
+    which would make the step look faster, so a non-zero word fails the run.
+    -> (ms per step, [ms per step of every repeat], launches per repeat, wall-clock start, end)"""
+    import torch
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    per_step, launches = [], 0
+    t0 = time.perf_counter()
+    for _ in range(max(1, args.repeats)):
+        barrier()
+        n0 = gb.gswa_launch_count()
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        barrier()
+        launches = gb.gswa_launch_count() - n0
+        check_status()                                   # raises on GSWA_ERR_DEVICE
+        per_step.append(max_over_ranks(e0.elapsed_time(e1)) / args.steps)
+    t1 = time.perf_counter()
+    return float(np.median(per_step)), per_step, int(launches), t0, t1
+
+
 def run_ours(args, cfg):
     import torch
     import torch.distributed as dist
@@ -284,41 +309,16 @@ def run_ours(args, cfg):
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
+    gb.gswa_scratch_status(desc, scratch)
     fused_peak = torch.cuda.max_memory_allocated() - mem0
     sampler = ClockSampler(local) if rank == 0 else None
     time.sleep(0.25 if rank == 0 else 0.0)
-    barrier()
-    n0 = gb.gswa_launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0 = time.perf_counter()
-    e0.record()
-    for _ in range(args.steps):
-        step()
-    e1.record()
-    barrier()
-    t1 = time.perf_counter()
-    launches = gb.gswa_launch_count() - n0
-    ms = e0.elapsed_time(e1)
+    ms_step, ms_repeats, launches, t0, t1 = timed_repeats(args, step, barrier, lambda: gb.gswa_scratch_status(desc, scratch), gb)
     clocks = sampler.stop(t0, t1) if sampler else None
-    ms = max_over_ranks(ms)
-    ms_step = ms / args.steps
     value = world * cfg.tokens / (ms_step * 1e-3)
 
     # per-kernel durations (CUDA events on the launching stream, separate pass so the timed region stays clean)
-    gb.gswa_profile_enable(True)
-    for _ in range(args.steps):
-        step()
-    torch.cuda.synchronize()
-    gb.gswa_profile_enable(False)
-    recs = gb.gswa_profile_read()
-    per = {}
-    for name, t in recs:
-        a = per.setdefault(name, [0, 0.0])
-        a[0] += 1
-        a[1] += t
-    total_ms = sum(v[1] for v in per.values())
-    kernels = {k: {"launches_per_step": v[0] / args.steps, "ms_per_step": v[1] / args.steps,
-                   "share": v[1] / total_ms} for k, v in sorted(per.items(), key=lambda kv: -kv[1][1])}
+    kernels = per_kernel_times(args, step, gb)
 
     # end to end through the host-buffer entry point
     hout = {"y": torch.empty(inp["x"].shape, dtype=tdt).pin_memory(), "dx": torch.empty(inp["x"].shape, dtype=tdt).pin_memory()}
@@ -336,7 +336,7 @@ def run_ours(args, cfg):
     for _ in range(2):
         step_host()
     barrier()
-    tt0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(e2e_steps):
         step_host()
@@ -384,7 +384,8 @@ def run_ours(args, cfg):
                    images, cfg.B, cfg.name, tokens, dt)}
 
     line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "repeats": len(ms_repeats),
+            "ms_per_step_repeats": [round(v, 5) for v in ms_repeats], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic", "config": dict(workload_config(cfg), flags=args.flags),
             "tflops": F * world / (ms_step * 1e-3) / 1e12,
             "layer_roofline": {"frac_burst": t_roof / (ms_step * 1e-3), "frac_sustained": t_roof_sus / (ms_step * 1e-3),
@@ -396,6 +397,111 @@ def run_ours(args, cfg):
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def per_kernel_times(args, step, gb):
+    """Per-kernel durations: CUDA events on the launching stream around every launch, in a separate pass so that
+    the timed region stays clean."""
+    import torch
+    gb.gswa_profile_enable(True)
+    for _ in range(args.steps):
+        step()
+    torch.cuda.synchronize()
+    gb.gswa_profile_enable(False)
+    per = {}
+    for name, t in gb.gswa_profile_read():
+        a = per.setdefault(name, [0, 0.0])
+        a[0] += 1
+        a[1] += t
+    total_ms = sum(v[1] for v in per.values())
+    return {k: {"launches_per_step": v[0] / args.steps, "ms_per_step": v[1] / args.steps, "share": v[1] / total_ms}
+            for k, v in sorted(per.items(), key=lambda kv: -kv[1][1])}
+
+
+def run_inference(args, cfg):
+    """Forward-only workloads: `cfg.layers` stacked layers with alternating group assignment and independent
+    weights, activations ping-ponging between two buffers, every call in inference mode (no carry is kept)."""
+    import torch
+    from paper_2409_06206_b200 import binding as gb
+    from paper_2409_06206_b200 import build as gbuild
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        gbuild.build()
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    barrier()
+    gb.lib()
+    tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    seeded = dataclass_replace(cfg, seed=cfg.seed + 1000 * rank)
+    mem0 = torch.cuda.memory_allocated()
+    torch.cuda.reset_peak_memory_stats()
+    x0 = torch.from_numpy(make_inputs(seeded, tensors=("x",))["x"]).to(tdt).cuda()
+    names = ("w_qkv", "b_qkv", "w_proj", "b_proj", "bias_table")
+    params = [{k: torch.from_numpy(v).to(tdt).cuda() for k, v in make_inputs(seeded, layer=l, tensors=names).items()}
+              for l in range(cfg.layers)]
+    descs = [gb.Desc.from_config(cfg, layer=l, flags=args.flags) for l in range(cfg.layers)]
+    infer_b = max(gb.gswa_workspace_query(d)[2] for d in descs)
+    scratch = torch.empty(max(infer_b, 16), dtype=torch.uint8, device="cuda")
+    bufs = [torch.empty_like(x0), torch.empty_like(x0)]
+
+    def step():
+        src = x0
+        for l in range(cfg.layers):
+            dst = bufs[l & 1]
+            p = params[l]
+            gb.gswa_forward(descs[l], src, p["w_qkv"], p["b_qkv"], p["w_proj"], p["b_proj"], p["bias_table"], dst, None, scratch)
+            src = dst
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    gb.gswa_scratch_status(descs[0], scratch)
+    peak = torch.cuda.max_memory_allocated() - mem0
+    sampler = ClockSampler(local) if rank == 0 else None
+    time.sleep(0.25 if rank == 0 else 0.0)
+    ms_step, ms_repeats, launches, t0, t1 = timed_repeats(args, step, barrier, lambda: gb.gswa_scratch_status(descs[0], scratch), gb)
+    clocks = sampler.stop(t0, t1) if sampler else None
+    kernels = per_kernel_times(args, step, gb)
+    if rank != 0:
+        return
+    pk, pk_src = peaks()
+    F = flops_per_token(cfg, backward=False) * cfg.tokens * cfg.layers
+    Bt = bytes_per_token(cfg, backward=False) * cfg.tokens * cfg.layers
+    t_roof = max(F / (pk["bf16_tflops"] * 1e12), Bt / (pk["hbm_gbs"] * 1e9))
+    t_roof_sus = max(F / (pk["bf16_tflops_sustained"] * 1e12), Bt / (pk["hbm_gbs"] * 1e9))
+    cpu = None
+    if world == 1 and not args.no_cpu:
+        # one layer of the stack on a 128 x 128 crop-sized draw of the same recipe: about 10 s of CPU work
+        small = dataclass_replace(cfg, H=128, W=128)
+        v, dt, tokens = time_oracle(small, 1)
+        cpu = {"value": v / cfg.layers, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
+               "sample": "one layer on a 128x128 image of the %s recipe (%d tokens) in %.1f s, numpy float64 forward; "
+                         "value = that rate / %d layers" % (cfg.name, tokens, dt, cfg.layers)}
+    line = {"metric": "GSWA fwd tokens/s through %d stacked layers" % cfg.layers,
+            "value": world * cfg.tokens / (ms_step * 1e-3), "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "repeats": len(ms_repeats),
+            "ms_per_step_repeats": [round(v, 5) for v in ms_repeats], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic", "config": dict(workload_config(cfg), flags=args.flags),
+            "token_layers_per_s": world * cfg.tokens * cfg.layers / (ms_step * 1e-3),
+            "tflops": F * world / (ms_step * 1e-3) / 1e12,
+            "layer_roofline": {"frac_burst": t_roof / (ms_step * 1e-3), "frac_sustained": t_roof_sus / (ms_step * 1e-3),
+                               "roofline_us": t_roof * 1e6, "alg_flops": F, "alg_bytes": Bt, "peaks": pk_src},
+            "roofline": dominant_roofline(cfg, kernels, pk, pk_src), "kernels": kernels, "gpu_launches": int(launches),
+            "e2e": None, "peak_mem": {"fused_peak_bytes": int(peak), "scratch_bytes": infer_b},
+            "cpu_baseline": cpu, "clocks": clocks}
+    print(json.dumps(line), flush=True)
 
 
 def dataclass_replace(cfg, **kw):
@@ -423,10 +529,10 @@ def kernel_cost(cfg: LayerConfig, name: str):
     return table.get(alias.get(name, name))
 
 
-# DRAM bytes per token of each kernel, dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture
-# on workload c3 (131072 tokens; traffic grows in proportion to the tokens) divided by its tokens.
-# None = not captured since the kernel last changed.  Source: profiles/.
-NCU_DRAM_BYTES_PER_TOKEN = {"attn_bwd": 314.09e6 / 131072}   # profiles/attn_bwd_c3_ncu.md
+# DRAM bytes per token of each kernel: dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of that
+# kernel on workload c3 (131072 tokens; traffic grows in proportion to the tokens) divided by its tokens.
+# A kernel is listed only while it is unchanged since its counters were taken (else `traffic` is null).
+NCU_DRAM_BYTES_PER_TOKEN = {"attn_bwd": 314.09e6 / 131072}
 
 
 def dominant_roofline(cfg, kernels, pk, pk_src):
@@ -465,7 +571,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="cM", choices=[k for k, c in CONFIGS.items() if c.backward])
+    ap.add_argument("--repeats", type=int, default=5, help="the K timed steps are measured this many times; the median is reported")
+    ap.add_argument("--workload", default="cM", choices=sorted(CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--flags", type=int, default=0, help="GSWA_FLAG_* bits for the layer descriptor (measured alternatives: "
                     "4 = fused QKV + forward attention, 8 = attention backward on tcgen05)")
@@ -475,6 +582,8 @@ def main():
     cfg = CONFIGS[args.workload]
     if args.impl == "reference":
         run_reference(args, cfg)
+    elif not cfg.backward:
+        run_inference(args, cfg)
     else:
         run_ours(args, cfg)
 

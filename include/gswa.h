@@ -15,18 +15,27 @@
  * pointer owned by the caller, 16-byte aligned, valid until the work enqueued
  * on `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream) has
  * finished.  Except where stated the library allocates no device memory and
- * keeps no state between calls.  Every function returns GSWA_OK (0) or a
- * negative gswa_status; argument errors are reported before anything is
- * enqueued; nothing throws, traps or asserts on the device.
+ * keeps no tensor state between calls.  What it does keep, per device and
+ * until the process exits: one internal non-blocking stream with three events
+ * (created on the first gswa_backward of a bf16 tensor-core layer; that call
+ * forks its two weight-gradient GEMMs onto it and joins it back into
+ * `cuda_stream` before returning, on every exit path, so the caller only ever
+ * orders against `cuda_stream`; concurrent gswa_backward calls on one device
+ * take turns enqueueing on it), the cached multiprocessor count, and the
+ * address of the built-in array of gswa_forward_static.  Every function returns
+ * GSWA_OK (0) or a negative gswa_status; argument errors are reported before
+ * anything is enqueued; nothing throws, traps or asserts on the device.
  *
  * Tensor conventions (the paper leaves them open):
  *   x, y, dy, dx      [B,H,W,C], C fastest.
  *   w_qkv             [3C, C] row-major (out, in); rows ordered q | k | v, head-major inside each.
- *   b_qkv             [3C] or NULL (= zeros).
- *   w_proj, b_proj    [C, C] (out, in), [C] or NULL.
+ *                     With narrowed projections (qk_dim, v_dim below): [2*heads*qk_dim + heads*v_dim, C].
+ *   b_qkv             [3C] (in general: one entry per row of w_qkv) or NULL (= zeros).
+ *   w_proj, b_proj    [C, C] (out, in) (in general [C, heads*v_dim]), [C] or NULL.
  *   bias_table        [(2M-1)^2, num_heads]; row (a_p-a_q+M-1)(2M-1) + (c_p-c_q+M-1) for query slot
  *                     (a_p,c_p) and key slot (a_q,c_q) of a window.
- *   q k^T is scaled by head_dim^-1/2; softmax runs over keys; the mask removes pairs (weight exactly 0).
+ *   q k^T is scaled by qk_dim^-1/2 (= head_dim^-1/2 by default); softmax runs over keys; the mask removes pairs
+ *   (weight exactly 0).
  *   cyclic shift by s: shifted[i',j'] = x[(i'+s) mod H, (j'+s) mod W].
  * All of x, y, dy, dx, weights, biases and the table have the element type
  * `dtype`; parameter gradients are always float32.
@@ -46,7 +55,7 @@ typedef enum gswa_status {
   GSWA_ERR_NULL = -1,        /* a required pointer is NULL                                  */
   GSWA_ERR_SHAPE = -2,       /* inconsistent sizes (H or W not a multiple of M, bad groups) */
   GSWA_ERR_ALIGN = -3,       /* a device pointer is not 16-byte aligned                     */
-  GSWA_ERR_UNSUPPORTED = -4, /* valid but not implemented (e.g. qk_dim != head_dim)         */
+  GSWA_ERR_UNSUPPORTED = -4, /* valid but not implemented (e.g. a window problem too large for one block) */
   GSWA_ERR_WORKSPACE = -5,   /* scratch / saved buffer too small                            */
   GSWA_ERR_CUDA = -6,        /* a CUDA runtime call or launch failed                        */
   GSWA_ERR_DEVICE = -7       /* a kernel gave up on a bounded internal wait (gswa_scratch_status) */
@@ -57,6 +66,8 @@ enum { GSWA_F32 = 0, GSWA_BF16 = 1 };
 enum {
   GSWA_FLAG_ACCUMULATE = 1u, /* add into the parameter gradients instead of overwriting them */
   GSWA_FLAG_GENERIC = 2u,    /* force the shape-generic CUDA-core kernels (no tensor-core fast path) */
+  /* (No flag asks for bitwise-reproducible reductions: the float32 parameter gradients are accumulated with
+   *  atomics on every path, see gswa_backward.) */
   GSWA_FLAG_FUSED_FWD = 4u,  /* tensor-core path: one kernel for QKV projection + forward attention (slower at C = 180; kept as a measured alternative) */
   GSWA_FLAG_TCGEN05_ATTN = 8u /* tensor-core path: attention backward on tcgen05 with TMEM accumulators instead of warp-level mma.sync (4 % slower at C = 180; kept as a measured alternative) */
 };
@@ -70,14 +81,18 @@ typedef struct gswa_desc {
   const int32_t* group_heads; /* host [G]; consecutive heads per group; sums to num_heads     */
   const int32_t* group_shift; /* host [G]; 0 <= s < M; 0 = plain windows, no mask             */
   int32_t dtype;              /* GSWA_F32 or GSWA_BF16                                        */
-  int32_t qk_dim, v_dim;      /* per-head widths; 0 = head_dim. Other values: GSWA_ERR_UNSUPPORTED */
+  int32_t qk_dim, v_dim;      /* per-head widths of q,k and of v (Sec. "Parameter Allocation": Q and K narrowed to
+                                 16 or 32 channels); 0 = head_dim = C / num_heads.  Other widths (<= 64) run on the
+                                 shape-generic kernels                                                            */
   uint32_t flags;             /* GSWA_FLAG_*                                                  */
 } gswa_desc;
 
 /* Buffer sizes for a layer description.
  *   saved_bytes          forward -> backward carry (projected q,k,v, attention output, row log-sum-exp).
  *   fwd_scratch_bytes    scratch of gswa_forward when `saved` is given.
- *   infer_scratch_bytes  scratch of gswa_forward when `saved` is NULL (the carry then lives in scratch).
+ *   infer_scratch_bytes  scratch of gswa_forward when `saved` is NULL (the carry then lives in scratch): a
+ *                        fourth size beside the three a training caller needs, so that an inference caller
+ *                        allocates one buffer instead of two.
  *   bwd_scratch_bytes    scratch of gswa_backward.
  * Any output pointer may be NULL. */
 int gswa_workspace_query(const gswa_desc* desc, size_t* saved_bytes, size_t* fwd_scratch_bytes,
@@ -112,6 +127,13 @@ int gswa_forward(const gswa_desc* desc, const void* x, const void* w_qkv, const 
 int gswa_forward_static(const gswa_desc* desc, const void* x, const void* w_qkv, const void* b_qkv,
                         const void* w_proj, const void* b_proj, const void* bias_table, void* y, void* cuda_stream);
 
+/* Device-side status of the last gswa_forward_static on the current device (the paper has no counterpart): what
+ * gswa_scratch_status is for caller-owned scratch, for the built-in array whose address the caller cannot name.
+ * Waits for `cuda_stream`; returns GSWA_OK or GSWA_ERR_DEVICE (y is then invalid).  Allocates nothing.  The
+ * array's address is looked up once per device and cached for the life of the process: after a cudaDeviceReset the
+ * cached address is stale, so a process that resets a device must not call the *_static functions on it again. */
+int gswa_static_status(void* cuda_stream);
+
 /* Backward pass (reverse mode of gswa_forward; the paper's stated target is the memory of
  * back-propagation).  `saved` is the buffer written by gswa_forward for the same desc and inputs; the weights must
  * be the ones that call was given (on the tensor-core path `saved` also carries the re-laid-out copies of them that
@@ -125,8 +147,9 @@ int gswa_backward(const gswa_desc* desc, const void* x, const void* w_qkv, const
                   float* db_qkv, float* dw_proj, float* db_proj, float* dbias_table, void* scratch,
                   size_t scratch_bytes, void* cuda_stream);
 
-/* Index maps of group `group`, computed on the device by the same routines the kernels use
- * (Sec. "Patch Embedding" window partition; cyclic shift and window mask of GSW-MSA).  All int32,
+/* Index maps of group `group`, computed on the device by the routines the shape-generic kernels use
+ * (Sec. "Patch Embedding" window partition; cyclic shift and window mask of GSW-MSA); gswa_debug_index_maps
+ * below exposes the arithmetic of the tensor-core kernels.  All int32,
  * any pointer may be NULL:
  *   win[H*W], slot[H*W], region[H*W]   per ORIGINAL token (i,j): window number in the shifted frame,
  *                                      slot inside it (row-major M x M), mask label 3*r(i')+r(j')
@@ -135,6 +158,24 @@ int gswa_backward(const gswa_desc* desc, const void* x, const void* w_qkv, const
  *   rel_index[M^2 * M^2]               bias-table row for (query slot, key slot). */
 int gswa_index_maps(const gswa_desc* desc, int32_t group, int32_t* win, int32_t* slot, int32_t* region,
                     int32_t* token_of, int32_t* rel_index, void* cuda_stream);
+
+/* Index maps of group `group` over the whole batch, computed by the arithmetic of the kernels that will run the
+ * layer: for a layer on the bf16 tensor-core path, by the window set-up and bias-row routines of its attention
+ * kernels; otherwise by the routines of gswa_index_maps.  For
+ * bit-exact comparison with the definition (Sec. "Patch Embedding"; shift and mask of GSW-MSA; Sec. "Learnable
+ * Relative Shifted Bias").  All int32 device pointers, any of them may be NULL:
+ *   win_id[B*H*W]        b * (H/M)(W/M) + window of every token in the shifted frame;
+ *   slot[H*W], region[H*W], rel_index[M^2 * M^2]   as in gswa_index_maps. */
+int gswa_debug_index_maps(const gswa_desc* desc, int32_t group, int32_t* win_id, int32_t* slot, int32_t* region,
+                          int32_t* rel_index, void* cuda_stream);
+
+/* Test hook for the device-side failure report (the paper has no counterpart): enqueues a one-block kernel that
+ * waits on a barrier nobody arrives on, gives up after about two thousand polls (well under a millisecond), sets the
+ * error word at the head of `scratch` exactly as a tensor-core kernel does when one of its bounded waits runs
+ * out, and returns normally.  gswa_scratch_status(desc, scratch) then reports GSWA_ERR_DEVICE; the next
+ * gswa_forward / gswa_backward on that scratch clears the word.  Nothing faults, traps or hangs.
+ * GSWA_ERR_UNSUPPORTED for layers off the tensor-core path (they keep no error word). */
+int gswa_debug_expire_wait(const gswa_desc* desc, void* scratch, void* cuda_stream);
 
 /* One training step on HOST buffers: copies x, the parameters and dy to the device arena, runs
  * gswa_forward + gswa_backward, copies y, dx and the parameter gradients back, and waits for the

@@ -29,6 +29,11 @@ are identities; masked weights are exactly 0; a closed form when Q,K and the
 table vanish; gradient invariants; central finite differences.  The paper
 prints no worked numerical example, so no printed values are pinned.
 
+Sec. "Parameter Allocation" (Q and K projections narrower than V): optional per-head
+widths `qk_dim`, `v_dim`; the scores are then scaled by qk_dim^-1/2.  Pinned by the same
+pins run at qk_dim != v_dim and by the identity "a narrow layer equals the full-width
+layer whose extra Q,K rows are zero and whose Q rows are rescaled by sqrt(d / qk_dim)".
+
 Conventions fixed where the paper is silent:
   x[B,H,W,C] channels last; w_qkv[3C,C] rows ordered [q|k|v], head-major
   inside each; y = x W^T + b; cyclic shift reads from +s
@@ -121,32 +126,46 @@ def _check(x, group_heads, group_shift, M):
     return B, H, W, C, nh, C // nh
 
 
-def forward(x, w_qkv, b_qkv, w_proj, b_proj, table, M, group_heads, group_shift, keep=True):
-    """y[B,H,W,C] and a cache for `backward`.  All arguments are converted to float64."""
+def _widths(d, qk_dim, v_dim):
+    """Per-head widths of Q,K and of V (Sec. "Parameter Allocation": Q and K may be narrower than V; both
+    default to the head dim C / heads)."""
+    return (int(qk_dim) if qk_dim else d), (int(v_dim) if v_dim else d)
+
+
+def forward(x, w_qkv, b_qkv, w_proj, b_proj, table, M, group_heads, group_shift, keep=True, qk_dim=None, v_dim=None):
+    """y[B,H,W,C] and a cache for `backward`.  All arguments are converted to float64.
+
+    With per-head widths dq = qk_dim and dv = v_dim (Sec. "Parameter Allocation"): w_qkv is
+    [2*heads*dq + heads*dv, C] with rows q | k | v (head-major inside each), w_proj is [C, heads*dv], and the
+    scores are scaled by dq^-1/2."""
     x = np.asarray(x, F64)
     w_qkv = np.asarray(w_qkv, F64)
     w_proj = np.asarray(w_proj, F64)
     table = np.asarray(table, F64)
     B, H, W, C, nh, d = _check(x, group_heads, group_shift, M)
-    b_qkv = np.zeros(3 * C, F64) if b_qkv is None else np.asarray(b_qkv, F64)
+    dq, dv = _widths(d, qk_dim, v_dim)
+    Cq, Cv = nh * dq, nh * dv
+    assert w_qkv.shape == (2 * Cq + Cv, C) and w_proj.shape == (C, Cv)
+    b_qkv = np.zeros(2 * Cq + Cv, F64) if b_qkv is None else np.asarray(b_qkv, F64)
     b_proj = np.zeros(C, F64) if b_proj is None else np.asarray(b_proj, F64)
     N = M * M
-    scale = float(d) ** -0.5
+    scale = float(dq) ** -0.5
 
     qkv = x @ w_qkv.T + b_qkv                                   # Eq. 6 projections
-    q = qkv[..., 0:C] * scale
-    k = qkv[..., C:2 * C]
-    v = qkv[..., 2 * C:3 * C]
+    q = qkv[..., 0:Cq] * scale
+    k = qkv[..., Cq:2 * Cq]
+    v = qkv[..., 2 * Cq:2 * Cq + Cv]
     rel = index_maps(H, W, M, 0)[3]
 
-    A = np.zeros((B, H, W, C), F64)
+    A = np.zeros((B, H, W, Cv), F64)
     groups = []
     h0 = 0
     for gh, s in zip(group_heads, group_shift):
-        ch = slice(h0 * d, (h0 + gh) * d)
-        qw = window_partition(cyclic_shift(q[..., ch], s), M).reshape(-1, N, gh, d)
-        kw = window_partition(cyclic_shift(k[..., ch], s), M).reshape(-1, N, gh, d)
-        vw = window_partition(cyclic_shift(v[..., ch], s), M).reshape(-1, N, gh, d)
+        chq = slice(h0 * dq, (h0 + gh) * dq)
+        ch = slice(h0 * dv, (h0 + gh) * dv)
+        qw = window_partition(cyclic_shift(q[..., chq], s), M).reshape(-1, N, gh, dq)
+        kw = window_partition(cyclic_shift(k[..., chq], s), M).reshape(-1, N, gh, dq)
+        vw = window_partition(cyclic_shift(v[..., ch], s), M).reshape(-1, N, gh, dv)
         S = np.einsum("nphd,nqhd->nhpq", qw, kw)
         S = S + table[rel][:, :, h0:h0 + gh].transpose(2, 0, 1)[None]      # bias B
         if s > 0:
@@ -156,9 +175,9 @@ def forward(x, w_qkv, b_qkv, w_proj, b_proj, table, M, group_heads, group_shift,
         Smax = S.max(axis=-1, keepdims=True)
         E = np.exp(S - Smax)
         P = E / E.sum(axis=-1, keepdims=True)
-        O = np.einsum("nhpq,nqhd->nphd", P, vw).reshape(-1, N, gh * d)
+        O = np.einsum("nhpq,nqhd->nphd", P, vw).reshape(-1, N, gh * dv)
         A[..., ch] = reverse_shift(window_reverse(O, M, B, H, W), s)        # concat of Eq. 7
-        groups.append((ch, s, qw, kw, vw, P) if keep else None)
+        groups.append((ch, s, qw, kw, vw, P, chq) if keep else None)
         h0 += gh
     y = A @ w_proj.T + b_proj                                               # W^P of Eq. 7
     cache = dict(x=x, w_qkv=w_qkv, w_proj=w_proj, table_shape=table.shape, M=M, group_heads=tuple(group_heads),
@@ -185,18 +204,19 @@ def backward(cache, dy):
     B, H, W, C = x.shape
     N = M * M
     dy2 = dy.reshape(-1, C)
-    dw_proj = dy2.T @ A.reshape(-1, C)
+    dw_proj = dy2.T @ A.reshape(-1, A.shape[-1])
     db_proj = dy2.sum(axis=0)
     dA = dy @ w_proj
 
-    dq = np.zeros((B, H, W, C), F64)
-    dk = np.zeros((B, H, W, C), F64)
-    dv = np.zeros((B, H, W, C), F64)
+    nh = int(sum(cache["group_heads"]))
+    wq, wv = cache["groups"][0][2].shape[-1], cache["groups"][0][4].shape[-1]   # per-head widths of q,k and of v
+    dq = np.zeros((B, H, W, nh * wq), F64)
+    dk = np.zeros((B, H, W, nh * wq), F64)
+    dv = np.zeros((B, H, W, nh * wv), F64)
     dtable = np.zeros(cache["table_shape"], F64)
     h0 = 0
-    for (ch, s, qw, kw, vw, P), gh in zip(cache["groups"], cache["group_heads"]):
-        d = qw.shape[-1]
-        dO = window_partition(cyclic_shift(dA[..., ch], s), M).reshape(-1, N, gh, d)
+    for (ch, s, qw, kw, vw, P, chq), gh in zip(cache["groups"], cache["group_heads"]):
+        dO = window_partition(cyclic_shift(dA[..., ch], s), M).reshape(-1, N, gh, wv)
         dvw = np.einsum("nhpq,nphd->nqhd", P, dO)
         dP = np.einsum("nphd,nqhd->nhpq", dO, vw)
         dS = P * (dP - (P * dP).sum(axis=-1, keepdims=True))                # softmax Jacobian
@@ -205,22 +225,24 @@ def backward(cache, dy):
         dSh = dS.sum(axis=0)                                                # [gh,N,N]
         for hh in range(gh):
             np.add.at(dtable[:, h0 + hh], rel.ravel(), dSh[hh].ravel())
-        for dst, src in ((dq, dqw), (dk, dkw), (dv, dvw)):
-            dst[..., ch] = reverse_shift(window_reverse(src.reshape(-1, N, gh * d), M, B, H, W), s)
+        for dst, src, sl, wd in ((dq, dqw, chq, wq), (dk, dkw, chq, wq), (dv, dvw, ch, wv)):
+            dst[..., sl] = reverse_shift(window_reverse(src.reshape(-1, N, gh * wd), M, B, H, W), s)
         h0 += gh
-    dqkv = np.concatenate([dq * scale, dk, dv], axis=-1).reshape(-1, 3 * C)
+    dqkv = np.concatenate([dq * scale, dk, dv], axis=-1).reshape(-1, nh * (2 * wq + wv))
     dw_qkv = dqkv.T @ x.reshape(-1, C)
     db_qkv = dqkv.sum(axis=0)
     dx = (dqkv @ w_qkv).reshape(B, H, W, C)
     return dict(dx=dx, dw_qkv=dw_qkv, db_qkv=db_qkv, dw_proj=dw_proj, db_proj=db_proj, dbias_table=dtable)
 
 
-def forward_backward_chunked(x, w_qkv, b_qkv, w_proj, b_proj, table, M, group_heads, group_shift, dy, chunk=4):
+def forward_backward_chunked(x, w_qkv, b_qkv, w_proj, b_proj, table, M, group_heads, group_shift, dy, chunk=4,
+                             qk_dim=None, v_dim=None):
     """Same results as forward + backward, walking the batch `chunk` images at a time to bound memory."""
     B = x.shape[0]
     ys, dxs, acc = [], [], None
     for b0 in range(0, B, chunk):
-        y, cache = forward(x[b0:b0 + chunk], w_qkv, b_qkv, w_proj, b_proj, table, M, group_heads, group_shift)
+        y, cache = forward(x[b0:b0 + chunk], w_qkv, b_qkv, w_proj, b_proj, table, M, group_heads, group_shift,
+                           qk_dim=qk_dim, v_dim=v_dim)
         g = backward(cache, dy[b0:b0 + chunk])
         ys.append(y)
         dxs.append(g.pop("dx"))
@@ -232,7 +254,7 @@ def forward_backward_chunked(x, w_qkv, b_qkv, w_proj, b_proj, table, M, group_he
 # --------------------------------------------------------------------------
 # forward, brute force over the whole image (no roll, no partition, no region labels)
 # --------------------------------------------------------------------------
-def bruteforce_forward(x, w_qkv, b_qkv, w_proj, b_proj, table, M, group_heads, group_shift):
+def bruteforce_forward(x, w_qkv, b_qkv, w_proj, b_proj, table, M, group_heads, group_shift, qk_dim=None, v_dim=None):
     """Masked global attention in original coordinates; pure loops, tiny inputs only.
 
     A shifted group cuts the image at rows/cols s + k*M.  Two tokens may attend
@@ -246,20 +268,22 @@ def bruteforce_forward(x, w_qkv, b_qkv, w_proj, b_proj, table, M, group_heads, g
     w_proj = np.asarray(w_proj, F64)
     table = np.asarray(table, F64)
     B, H, W, C, nh, d = _check(x, group_heads, group_shift, M)
-    b_qkv = np.zeros(3 * C, F64) if b_qkv is None else np.asarray(b_qkv, F64)
+    dq, dv = _widths(d, qk_dim, v_dim)
+    Cq, Cv = nh * dq, nh * dv
+    b_qkv = np.zeros(2 * Cq + Cv, F64) if b_qkv is None else np.asarray(b_qkv, F64)
     b_proj = np.zeros(C, F64) if b_proj is None else np.asarray(b_proj, F64)
     head_shift = [s for gh, s in zip(group_heads, group_shift) for _ in range(gh)]
-    A = np.zeros((B, H, W, C), F64)
+    A = np.zeros((B, H, W, Cv), F64)
     for b in range(B):
         tok = x[b].reshape(H * W, C)
         for h in range(nh):
             s = head_shift[h]
-            wq = w_qkv[h * d:(h + 1) * d]
-            wk = w_qkv[C + h * d:C + (h + 1) * d]
-            wv = w_qkv[2 * C + h * d:2 * C + (h + 1) * d]
-            q = tok @ wq.T + b_qkv[h * d:(h + 1) * d]
-            k = tok @ wk.T + b_qkv[C + h * d:C + (h + 1) * d]
-            v = tok @ wv.T + b_qkv[2 * C + h * d:2 * C + (h + 1) * d]
+            rq = slice(h * dq, (h + 1) * dq)
+            rk = slice(Cq + h * dq, Cq + (h + 1) * dq)
+            rv = slice(2 * Cq + h * dv, 2 * Cq + (h + 1) * dv)
+            q = tok @ w_qkv[rq].T + b_qkv[rq]
+            k = tok @ w_qkv[rk].T + b_qkv[rk]
+            v = tok @ w_qkv[rv].T + b_qkv[rv]
             for p in range(H * W):
                 ip, jp = divmod(p, W)
                 logits, keys = [], []
@@ -268,10 +292,10 @@ def bruteforce_forward(x, w_qkv, b_qkv, w_proj, b_proj, table, M, group_heads, g
                     if (ip - s) // M != (ir - s) // M or (jp - s) // M != (jr - s) // M:
                         continue
                     row = (ip - ir + M - 1) * (2 * M - 1) + (jp - jr + M - 1)
-                    logits.append(float(q[p] @ k[r]) / np.sqrt(d) + table[row, h])
+                    logits.append(float(q[p] @ k[r]) / np.sqrt(dq) + table[row, h])
                     keys.append(r)
                 logits = np.array(logits)
                 wgt = np.exp(logits - logits.max())
                 wgt /= wgt.sum()
-                A[b, ip, jp, h * d:(h + 1) * d] = wgt @ v[keys]
+                A[b, ip, jp, h * dv:(h + 1) * dv] = wgt @ v[keys]
     return A @ w_proj.T + b_proj

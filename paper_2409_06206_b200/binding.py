@@ -19,8 +19,8 @@ FLAG_ACCUMULATE, FLAG_GENERIC, FLAG_FUSED_FWD, FLAG_TCGEN05_ATTN = 1, 2, 4, 8
 
 STATIC_SCRATCH_BYTES = 16 << 20
 
-EXPORTS = ("gswa_workspace_query", "gswa_forward", "gswa_forward_static", "gswa_backward", "gswa_index_maps", "gswa_step_host",
-           "gswa_scratch_status", "gswa_profile_enable", "gswa_profile_read", "gswa_launch_count", "gswa_status_string")
+EXPORTS = ("gswa_workspace_query", "gswa_forward", "gswa_forward_static", "gswa_static_status", "gswa_backward",
+           "gswa_index_maps", "gswa_debug_index_maps", "gswa_debug_expire_wait", "gswa_step_host", "gswa_scratch_status", "gswa_profile_enable", "gswa_profile_read", "gswa_launch_count", "gswa_status_string")
 
 
 class GswaError(RuntimeError):
@@ -58,7 +58,7 @@ class Desc:
         from .inputs import layer_groups
         gh, gs = layer_groups(cfg, layer)
         return cls(cfg.B if batch is None else batch, cfg.H, cfg.W, cfg.C, cfg.num_heads, cfg.window, gh, gs,
-                   cfg.dtype, flags)
+                   cfg.dtype, flags, getattr(cfg, "qk_dim", 0), getattr(cfg, "v_dim", 0))
 
     def with_flags(self, flags: int) -> "Desc":
         B, H, W, C_ = self.shape
@@ -88,6 +88,12 @@ def lib() -> C.CDLL:
         L.gswa_step_host.argtypes = [dp] + [vp] * 15 + [sz, szp, vp]
         L.gswa_scratch_status.argtypes = [dp, vp, vp]
         L.gswa_scratch_status.restype = C.c_int
+        L.gswa_static_status.argtypes = [vp]
+        L.gswa_static_status.restype = C.c_int
+        L.gswa_debug_index_maps.argtypes = [dp, C.c_int32] + [vp] * 5
+        L.gswa_debug_index_maps.restype = C.c_int
+        L.gswa_debug_expire_wait.argtypes = [dp, vp, vp]
+        L.gswa_debug_expire_wait.restype = C.c_int
         L.gswa_profile_enable.argtypes = [C.c_int]
         L.gswa_profile_read.argtypes = [C.c_int32, C.c_char_p, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
         L.gswa_profile_enable.restype = C.c_int
@@ -164,6 +170,21 @@ def gswa_backward(desc: Desc, x, w_qkv, b_qkv, w_proj, bias_table, saved, dy, dx
 def gswa_index_maps(desc: Desc, group: int, win, slot, region, token_of, rel_index, stream=None) -> None:
     _check(lib().gswa_index_maps(C.byref(desc.c), group, _ptr(win), _ptr(slot), _ptr(region), _ptr(token_of),
                                  _ptr(rel_index), _stream(stream)))
+
+
+def gswa_debug_index_maps(desc: Desc, group: int, win_id, slot, region, rel_index, stream=None) -> None:
+    _check(lib().gswa_debug_index_maps(C.byref(desc.c), group, _ptr(win_id), _ptr(slot), _ptr(region), _ptr(rel_index),
+                                       _stream(stream)))
+
+
+def gswa_debug_expire_wait(desc: Desc, scratch, stream=None) -> None:
+    """Test hook: makes a bounded device-side wait run out on purpose (sets the error word of `scratch`)."""
+    _check(lib().gswa_debug_expire_wait(C.byref(desc.c), _ptr(scratch), _stream(stream)))
+
+
+def gswa_static_status(stream=None) -> None:
+    """Waits for the stream and raises GswaError(-7) if the last gswa_forward_static on this device gave up a wait."""
+    _check(lib().gswa_static_status(_stream(stream)))
 
 
 def gswa_step_host_arena_bytes(desc: Desc) -> int:

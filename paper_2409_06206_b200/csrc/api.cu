@@ -41,6 +41,19 @@ KernelScope::~KernelScope() {
 
 bool profiling_enabled() { return g_prof_on; }
 
+int device_sm_count() {
+  constexpr int kMaxDev = 64;
+  static std::atomic<int> cache[kMaxDev];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) { (void)cudaGetLastError(); return 148; }
+  int n = cache[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) { (void)cudaGetLastError(); n = 148; }
+    cache[dev].store(n, std::memory_order_relaxed);
+  }
+  return n;
+}
+
 int check_launch() {
   const cudaError_t e = cudaGetLastError();
   if (e == cudaSuccess) return GSWA_OK;
@@ -56,6 +69,8 @@ static int cuda_rc(cudaError_t e) {
 }
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+constexpr size_t kMaxBlockSmem = 227 * 1024;   // opt-in dynamic shared memory of one block on sm_100
 
 int make_plan(const gswa_desc* desc, Plan* p) {
   if (desc == nullptr || p == nullptr) return GSWA_ERR_NULL;
@@ -79,9 +94,11 @@ int make_plan(const gswa_desc* desc, Plan* p) {
     sum += p->gh[g];
   }
   if (sum != p->nh) return GSWA_ERR_SHAPE;
-  if ((desc->qk_dim != 0 && desc->qk_dim != p->d) || (desc->v_dim != 0 && desc->v_dim != p->d))
-    return GSWA_ERR_UNSUPPORTED;
-  if (p->N > 144 || p->d > 64) return GSWA_ERR_UNSUPPORTED;
+  if (desc->qk_dim < 0 || desc->v_dim < 0) return GSWA_ERR_SHAPE;
+  p->dqk = desc->qk_dim ? desc->qk_dim : p->d;
+  p->dv = desc->v_dim ? desc->v_dim : p->d;
+  p->Cq = p->nh * p->dqk; p->Cv = p->nh * p->dv; p->Cqkv = 2 * p->Cq + p->Cv;
+  if (p->N > 144 || p->dqk > 64 || p->dv > 64) return GSWA_ERR_UNSUPPORTED;
   const long long T = (long long)p->B * p->H * p->W;
   if (T * 3 * p->C >= (1LL << 40) || T >= (1LL << 31) / 2) return GSWA_ERR_UNSUPPORTED;
   p->T = T;
@@ -91,13 +108,17 @@ int make_plan(const gswa_desc* desc, Plan* p) {
   // generic path: saved = qkv[T,3C] | A[T,C] | L[T,nh] (float)
   const size_t es = (size_t)p->esize;
   p->off_qkv = 0;
-  p->off_A = align_up((size_t)T * 3 * p->C * es, 256);
-  p->off_L = p->off_A + align_up((size_t)T * p->C * es, 256);
+  p->off_A = align_up((size_t)T * p->Cqkv * es, 256);
+  p->off_L = p->off_A + align_up((size_t)T * p->Cv * es, 256);
   p->saved_bytes = p->off_L + align_up((size_t)T * p->nh * sizeof(float), 256);
   p->fwd_scratch = 0;
   p->infer_scratch = p->saved_bytes;
-  p->bwd_scratch = align_up((size_t)T * 4 * p->C * es, 256);  // dA[T,C] | dqkv[T,3C]
-  if (fast_path_ok(*p)) fast_plan_sizes(p);
+  p->bwd_scratch = align_up((size_t)T * (p->Cv + p->Cqkv) * es, 256);  // dA[T,Cv] | dqkv[T,Cqkv]
+  if (fast_path_ok(*p)) {
+    fast_plan_sizes(p);
+  } else if (generic_attn_fwd_smem(*p) > kMaxBlockSmem || generic_attn_bwd_smem(*p) > kMaxBlockSmem) {
+    return GSWA_ERR_UNSUPPORTED;   // one (window, head) problem must fit the shared memory of one block
+  }
   return GSWA_OK;
 }
 
@@ -110,6 +131,7 @@ static __device__ __align__(256) unsigned char g_static_scratch[GSWA_STATIC_SCRA
 constexpr int kMaxDevices = 64;
 static std::mutex g_static_mu;
 static void* g_static_ptr[kMaxDevices] = {};
+static bool g_static_has_word[kMaxDevices] = {};   // the last gswa_forward_static on the device left an error word at the head of the array
 
 // Device address of g_static_scratch on the current device (looked up once per device).
 static int static_scratch(void** out) {
@@ -179,6 +201,13 @@ int gswa_forward_static(const gswa_desc* desc, const void* x, const void* w_qkv,
   if (p.infer_scratch > (size_t)GSWA_STATIC_SCRATCH_BYTES) return GSWA_ERR_WORKSPACE;   // layer too large for the built-in array
   void* scratch = nullptr;
   if ((rc = static_scratch(&scratch))) return rc;
+  {
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices) {
+      std::lock_guard<std::mutex> lk(g_static_mu);
+      g_static_has_word[dev] = p.fast && p.T > 0;          // the generic kernels have no bounded waits and keep no word
+    }
+  }
   // same path as gswa_forward with saved == NULL; the device error word at the head of the scratch
   // is cleared by that path on every call
   return gswa_forward(desc, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, y, nullptr, scratch,
@@ -204,11 +233,11 @@ int gswa_backward(const gswa_desc* desc, const void* x, const void* w_qkv, const
   {
     // one launch zeroes the parameter gradients (unless they accumulate) and, on the tensor-core path, the error
     // word at the head of the scratch buffer
-    const size_t C = (size_t)p.C, nrel = (size_t)(2 * p.M - 1) * (2 * p.M - 1);
+    const size_t C = (size_t)p.C, Q = (size_t)p.Cqkv, Cv = (size_t)p.Cv, nrel = (size_t)(2 * p.M - 1) * (2 * p.M - 1);
     const bool z = !(p.flags & GSWA_FLAG_ACCUMULATE);
     float* const ptrs[6] = {z ? dw_qkv : nullptr, z ? db_qkv : nullptr, z ? dw_proj : nullptr, z ? db_proj : nullptr,
                             z ? dbias_table : nullptr, p.fast && p.T > 0 ? static_cast<float*>(scratch) : nullptr};
-    const long long counts[6] = {(long long)(3 * C * C), (long long)(3 * C), (long long)(C * C), (long long)C,
+    const long long counts[6] = {(long long)(Q * C), (long long)Q, (long long)(C * Cv), (long long)C,
                                  (long long)(nrel * p.nh), 64};
     if ((rc = launch_zero(ptrs, counts, 6, st))) return rc;
   }
@@ -229,6 +258,47 @@ int gswa_index_maps(const gswa_desc* desc, int32_t group, int32_t* win, int32_t*
   return launch_index_maps(p, group, win, slot, region, token_of, rel_index, reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
+int gswa_debug_index_maps(const gswa_desc* desc, int32_t group, int32_t* win_id, int32_t* slot, int32_t* region,
+                          int32_t* rel_index, void* cuda_stream) {
+  Plan p;
+  int rc = make_plan(desc, &p);
+  if (rc) return rc;
+  if (group < 0 || group >= p.G) return GSWA_ERR_SHAPE;
+  if (p.T == 0) return GSWA_OK;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (p.fast) return fast_index_maps(p, group, win_id, slot, region, rel_index, st);
+  if ((slot || region || rel_index) && (rc = launch_index_maps(p, group, nullptr, slot, region, nullptr, rel_index, st))) return rc;
+  return win_id ? launch_batch_window_ids(p, group, win_id, st) : GSWA_OK;
+}
+
+int gswa_debug_expire_wait(const gswa_desc* desc, void* scratch, void* cuda_stream) {
+  Plan p;
+  const int rc = make_plan(desc, &p);
+  if (rc) return rc;
+  if (!p.fast) return GSWA_ERR_UNSUPPORTED;        // only the tensor-core path keeps an error word in its scratch
+  if (scratch == nullptr) return GSWA_ERR_NULL;
+  if (misaligned(scratch)) return GSWA_ERR_ALIGN;
+  return launch_wait_timeout(static_cast<int*>(scratch), reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int gswa_static_status(void* cuda_stream) {
+  void* scratch = nullptr;
+  int rc = static_scratch(&scratch);
+  if (rc) return rc;
+  {
+    int dev = 0;
+    if ((rc = cuda_rc(cudaGetDevice(&dev)))) return rc;
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    if (dev < 0 || dev >= kMaxDevices || !g_static_has_word[dev]) return GSWA_OK;
+  }
+  int word = 0;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  rc = cuda_rc(cudaMemcpyAsync(&word, scratch, sizeof(int), cudaMemcpyDeviceToHost, st));
+  if (rc == GSWA_OK) rc = cuda_rc(cudaStreamSynchronize(st));
+  if (rc) return rc;
+  return word == 0 ? GSWA_OK : GSWA_ERR_DEVICE;
+}
+
 int gswa_step_host(const gswa_desc* desc, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
                    const void* b_proj, const void* bias_table, const void* dy, void* y, void* dx, float* dw_qkv,
                    float* db_qkv, float* dw_proj, float* db_proj, float* dbias_table, void* arena,
@@ -236,15 +306,16 @@ int gswa_step_host(const gswa_desc* desc, const void* x, const void* w_qkv, cons
   Plan p;
   int rc = make_plan(desc, &p);
   if (rc) return rc;
-  const size_t es = (size_t)p.esize, C = (size_t)p.C, nrel = (size_t)(2 * p.M - 1) * (2 * p.M - 1);
+  const size_t es = (size_t)p.esize, C = (size_t)p.C, Q = (size_t)p.Cqkv, Cv = (size_t)p.Cv;
+  const size_t nrel = (size_t)(2 * p.M - 1) * (2 * p.M - 1);
   const size_t act = align_up((size_t)p.T * C * es, 256);
   // arena layout
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
   const size_t o_x = take(act), o_dy = take(act), o_y = take(act), o_dx = take(act);
-  const size_t o_wqkv = take(3 * C * C * es), o_bqkv = take(3 * C * es), o_wproj = take(C * C * es);
+  const size_t o_wqkv = take(Q * C * es), o_bqkv = take(Q * es), o_wproj = take(C * Cv * es);
   const size_t o_bproj = take(C * es), o_tab = take(nrel * p.nh * es);
-  const size_t o_dwqkv = take(3 * C * C * 4), o_dbqkv = take(3 * C * 4), o_dwproj = take(C * C * 4);
+  const size_t o_dwqkv = take(Q * C * 4), o_dbqkv = take(Q * 4), o_dwproj = take(C * Cv * 4);
   const size_t o_dbproj = take(C * 4), o_dtab = take(nrel * p.nh * 4);
   const size_t o_saved = take(p.saved_bytes);
   const size_t scr = p.fwd_scratch > p.bwd_scratch ? p.fwd_scratch : p.bwd_scratch;
@@ -264,10 +335,10 @@ int gswa_step_host(const gswa_desc* desc, const void* x, const void* w_qkv, cons
   auto d2h = [&](void* dst, size_t o, size_t bytes) {
     return cuda_rc(cudaMemcpyAsync(dst, a + o, bytes, cudaMemcpyDeviceToHost, st));
   };
-  if ((rc = h2d(o_x, x, act_b)) || (rc = h2d(o_dy, dy, act_b)) || (rc = h2d(o_wqkv, w_qkv, 3 * C * C * es)) ||
-      (rc = h2d(o_wproj, w_proj, C * C * es)) || (rc = h2d(o_tab, bias_table, nrel * p.nh * es)))
+  if ((rc = h2d(o_x, x, act_b)) || (rc = h2d(o_dy, dy, act_b)) || (rc = h2d(o_wqkv, w_qkv, Q * C * es)) ||
+      (rc = h2d(o_wproj, w_proj, C * Cv * es)) || (rc = h2d(o_tab, bias_table, nrel * p.nh * es)))
     return rc;
-  if (b_qkv && (rc = h2d(o_bqkv, b_qkv, 3 * C * es))) return rc;
+  if (b_qkv && (rc = h2d(o_bqkv, b_qkv, Q * es))) return rc;
   if (b_proj && (rc = h2d(o_bproj, b_proj, C * es))) return rc;
   rc = gswa_forward(desc, a + o_x, a + o_wqkv, b_qkv ? a + o_bqkv : nullptr, a + o_wproj, b_proj ? a + o_bproj : nullptr,
                     a + o_tab, a + o_y, a + o_saved, a + o_scr, scr, cuda_stream);
@@ -278,8 +349,8 @@ int gswa_step_host(const gswa_desc* desc, const void* x, const void* w_qkv, cons
                      a + o_dy, a + o_dx, (float*)(a + o_dwqkv), (float*)(a + o_dbqkv), (float*)(a + o_dwproj),
                      (float*)(a + o_dbproj), (float*)(a + o_dtab), a + o_scr, scr, cuda_stream);
   if (rc) return rc;
-  if ((rc = d2h(y, o_y, act_b)) || (rc = d2h(dx, o_dx, act_b)) || (rc = d2h(dw_qkv, o_dwqkv, 3 * C * C * 4)) ||
-      (rc = d2h(db_qkv, o_dbqkv, 3 * C * 4)) || (rc = d2h(dw_proj, o_dwproj, C * C * 4)) ||
+  if ((rc = d2h(y, o_y, act_b)) || (rc = d2h(dx, o_dx, act_b)) || (rc = d2h(dw_qkv, o_dwqkv, Q * C * 4)) ||
+      (rc = d2h(db_qkv, o_dbqkv, Q * 4)) || (rc = d2h(dw_proj, o_dwproj, C * Cv * 4)) ||
       (rc = d2h(db_proj, o_dbproj, C * 4)) || (rc = d2h(dbias_table, o_dtab, nrel * p.nh * 4)))
     return rc;
   return cuda_rc(cudaStreamSynchronize(st));

@@ -231,13 +231,18 @@ __device__ __forceinline__ WinCtx window_setup(const FastGeom& g, int s, long lo
 
 // The scores start from the relative-position bias (the MMAs then accumulate q k^T on top of it: no separate
 // addition); q and the table are already scaled by log2(e), the scores are in the log2 domain throughout.
-__device__ __forceinline__ void bias_init(float (*s)[4], const float2* tab2, int p0, int t) {
+// Bias-table row of query slot p0 against key slot 8*j + 2*t (the first of a thread's two key columns in key
+// block j of the mma fragment).  Key 8*j + 2*t + 1 uses row - 1, query p0 + 8 (next window row) uses row + 15.
+__device__ __forceinline__ int frag_bias_row(int p0, int t, int j) {
   const int pa0 = p0 >> 3, pc0 = p0 & 7;   // rows p0 and p0 + 8: same column in the window, next row
+  return (pa0 - j + 7) * 15 + (pc0 - 2 * t + 7);
+}
+__device__ __forceinline__ void bias_init(float (*s)[4], const float2* tab2, int p0, int t) {
   // a thread's two columns of a key block are neighbours in the table: entry r of the pair table holds
   // (table[r], table[r - 1]), so one 8-byte load fills two accumulators
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    const int r = (pa0 - j + 7) * 15 + (pc0 - 2 * t + 7);
+    const int r = frag_bias_row(p0, t, j);
     const float2 a = tab2[r], b = tab2[r + 15];
     s[j][0] = a.x; s[j][1] = a.y; s[j][2] = b.x; s[j][3] = b.y;
   }

@@ -121,7 +121,7 @@ GrShape gr_shape(const Plan& p, int which) {
   // dW_qkv: x is copied once for two M blocks of dqkv; dW_proj: two M blocks per CTA measured slower (fewer TMA stages)
   g.mbpc = which && 2 * g.NP <= 512 ? 2 : 1;
   const int mblocks = ((g.M + 127) / 128 + g.mbpc - 1) / g.mbpc;
-  const long long ns = 148 / mblocks, cap = (p.T + 63) / 64;
+  const long long ns = device_sm_count() / mblocks, cap = (p.T + 63) / 64;
   g.nsplit = (int)(ns < cap ? (ns < 1 ? 1 : ns) : cap);
   return g;
 }
@@ -169,6 +169,7 @@ BwdScratch bwd_layout(const Plan& p) {
 
 bool fast_path_ok(const Plan& p) {
   if (p.dtype != GSWA_BF16 || (p.flags & GSWA_FLAG_GENERIC)) return false;
+  if (p.dqk != p.d || p.dv != p.d) return false;             // narrowed Q/K projections run on the shape-generic kernels
   if (p.M != 8 || p.d > 32 || (p.d & 1) || (p.C & 3) || p.C > 252 || p.G > 4) return false;
   if (p.nh * (p.d <= 16 ? 16 : 32) < 64) return false;       // padded rows must fill one TMA box of 64 columns
   if (p.T >= (1LL << 30) / 4) return false;
@@ -201,6 +202,10 @@ void fast_plan_sizes(Plan* p) {
   p->fwd_scratch = fwd_layout(*p, units, nu, tp).total;
   p->infer_scratch = p->fwd_scratch + p->saved_bytes;
   p->bwd_scratch = bwd_layout(*p).total;
+}
+
+int fast_index_maps(const Plan& p, int group, int32_t* win_id, int32_t* slot, int32_t* region, int32_t* rel, cudaStream_t st) {
+  return launch_fast_index_maps(make_geom(p), p.gs[group], win_id, slot, region, rel, st);
 }
 
 // A second stream per device for the two weight-gradient GEMMs of the backward pass.  Nothing downstream reads
@@ -396,27 +401,67 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
   float* dummy = reinterpret_cast<float*>(sc + bs.dummy);      // (the error word was zeroed together with the gradients)
 
   int rc = GSWA_OK;
+  const BwdImages bi = bwd_images(p, units, nu, tx);          // built by the forward call
+  const unsigned char* bimg = reinterpret_cast<const unsigned char*>(sv + p.off_bimg);
+
+  // ---- everything that can fail on the host (tensor maps) comes first: once the side stream has been forked off,
+  // the only remaining failures are launch errors, and those still pass through the join below
+  GRLaunch grp{}, grx{};
+  GTLaunch gt{};
+  AttnLaunch al{};
+  const bool want_dwproj = dw_proj || db_proj, want_dwqkv = dw_qkv || db_qkv;
+  if (want_dwproj && (rc = make_tmap(&grp.tm, A, p.T, p.Ap, 64))) return rc;
+  if (dx && (rc = make_tmap(&gt.tmA, dqkv, p.T, 3 * p.Ap, 128))) return rc;
+  if (want_dwqkv && (rc = make_tmap(&grx.tm, dqkv, p.T, 3 * p.Ap, 64))) return rc;
+  attn_units(p, geo, units, nu, &al);
+  bool one_head_units = true;
+  for (int i = 0; i < al.nunits; ++i) one_head_units = one_head_units && al.u[i].nheads == 1;
+  const bool tc_attn = one_head_units && (p.flags & GSWA_FLAG_TCGEN05_ATTN);
+  if (tc_attn) {
+    if ((rc = make_tmap_window(&al.tm_out, dqkv, (long long)p.B * p.H, p.W, 3 * p.Ap, p.dp, 8, 8, true))) return rc;
+    // A window of a shifted group that wraps around the image edge is stored as four boxes.  Their shared-
+    // memory sources must start on 128-byte boundaries, which an even shift guarantees; units with another
+    // shift store such windows row by row.
+    al.wrap_s = 0;
+    for (int i = 0; i < al.nunits && al.wrap_s == 0; ++i)
+      if (al.u[i].s > 0 && al.u[i].s % 2 == 0) al.wrap_s = al.u[i].s;
+    if (al.wrap_s > 0) {
+      const int e = 8 - al.wrap_s, s = al.wrap_s;
+      for (int k = 0; k < 4; ++k)
+        if ((rc = make_tmap_window(&al.tm_wrap[k], dqkv, (long long)p.B * p.H, p.W, 3 * p.Ap, p.dp, (k & 1) ? s : e, (k & 2) ? s : e, false)))
+          return rc;
+    }
+  }
+
   // the weight-gradient GEMMs go to the side stream (not while kernels are being timed one by one)
   SideStream* ss = profiling_enabled() ? nullptr : side_stream();
   std::unique_lock<std::mutex> ss_lock;
   if (ss) ss_lock = std::unique_lock<std::mutex>(ss->use);
+  if (ss && (cudaEventRecord(ss->fork1, st) != cudaSuccess || cudaStreamWaitEvent(ss->s, ss->fork1, 0) != cudaSuccess)) {
+    (void)cudaGetLastError();
+    ss = nullptr;                                             // nothing was forked: stay on the caller's stream
+  }
   cudaStream_t s2 = ss ? ss->s : st;
-  if (ss && (cudaEventRecord(ss->fork1, st) != cudaSuccess || cudaStreamWaitEvent(s2, ss->fork1, 0) != cudaSuccess)) return check_launch();
-  const BwdImages bi = bwd_images(p, units, nu, tx);          // built by the forward call
-  const unsigned char* bimg = reinterpret_cast<const unsigned char*>(sv + p.off_bimg);
+  // From here on every exit joins the side stream back into the caller's stream: whatever was enqueued there is
+  // ordered before anything the caller enqueues next (and a stream capture is not left with an open fork).
+  auto finish = [&](int code) {
+    if (ss && (cudaEventRecord(ss->join, s2) != cudaSuccess || cudaStreamWaitEvent(st, ss->join, 0) != cudaSuccess)) {
+      const int jrc = check_launch();
+      return code ? code : jrc;
+    }
+    return code;
+  };
 
-  if (dw_proj || db_proj) {
+  if (want_dwproj) {
     // dW^P = dy^T A (A fetched by TMA); db^P rides on the ones column of A when the head dim is padded
-    GRLaunch gr{};
-    if ((rc = make_tmap(&gr.tm, A, p.T, p.Ap, 64))) return rc;
-    gr.tma_is_L = 0;
-    gr.P = (const bf*)dy; gr.ldp = p.C; gr.pvalid = p.C;
+    grp.tma_is_L = 0;
+    grp.P = (const bf*)dy; grp.ldp = p.C; grp.pvalid = p.C;
     const GrShape gs = gr_shape(p, 0);
-    gr.Ap = p.Ap; gr.dp = p.dp; gr.d = p.d; gr.C = p.C; gr.M = gs.M; gr.rows = p.T;
-    gr.NP = gs.NP; gr.mbpc = gs.mbpc; gr.nsplit = gs.nsplit;
-    gr.out = dw_proj ? dw_proj : dummy; gr.colsum = p.d < p.dp ? db_proj : nullptr; gr.err = err;
-    if ((rc = launch_gr(gr, s2, "dwproj_gemm"))) return rc;
-    if (db_proj && p.d == p.dp && (rc = launch_colsum_bf16((const bf*)dy, p.T, p.C, p.C, db_proj, s2))) return rc;
+    grp.Ap = p.Ap; grp.dp = p.dp; grp.d = p.d; grp.C = p.C; grp.M = gs.M; grp.rows = p.T;
+    grp.NP = gs.NP; grp.mbpc = gs.mbpc; grp.nsplit = gs.nsplit;
+    grp.out = dw_proj ? dw_proj : dummy; grp.colsum = p.d < p.dp ? db_proj : nullptr; grp.err = err;
+    if ((rc = launch_gr(grp, s2, "dwproj_gemm"))) return finish(rc);
+    if (db_proj && p.d == p.dp && (rc = launch_colsum_bf16((const bf*)dy, p.T, p.C, p.C, db_proj, s2))) return finish(rc);
   }
 
   // (dW^P runs first so that the dO tiles written next are still in L2 when the attention kernel reads them)
@@ -434,59 +479,36 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
     w.win_stride = (long long)p.gh[u.g] * 64 * p.dp;
     w.nchunks = 1; w.cw = u.nheads * p.dp; w.q_every3 = 0; w.qscale = 1.f;
   }
-  if ((rc = launch_gw(gw, nu, p.Cp, p.dp, st, "dattn_gemm"))) return rc;
+  if ((rc = launch_gw(gw, nu, p.Cp, p.dp, st, "dattn_gemm"))) return finish(rc);
 
-  AttnLaunch al{};
-  attn_units(p, geo, units, nu, &al);
   al.qkv = qkv; al.table = (const bf*)table; al.Lt = const_cast<float*>(Lt); al.dO = dO; al.dqkv = dqkv;
   al.dtable = dtable; al.scale = 1.0f / sqrtf((float)p.d); al.err = err;
-  bool one_head_units = true;
-  for (int i = 0; i < al.nunits; ++i) one_head_units = one_head_units && al.u[i].nheads == 1;
-  if (one_head_units && (p.flags & GSWA_FLAG_TCGEN05_ATTN)) {
-    if ((rc = make_tmap_window(&al.tm_out, dqkv, (long long)p.B * p.H, p.W, 3 * p.Ap, p.dp, 8, 8, true))) return rc;
-    // A window of a shifted group that wraps around the image edge is stored as four boxes.  Their shared-
-    // memory sources must start on 128-byte boundaries, which an even shift guarantees; units with another
-    // shift store such windows row by row.
-    al.wrap_s = 0;
-    for (int i = 0; i < al.nunits && al.wrap_s == 0; ++i)
-      if (al.u[i].s > 0 && al.u[i].s % 2 == 0) al.wrap_s = al.u[i].s;
-    if (al.wrap_s > 0) {
-      const int e = 8 - al.wrap_s, s = al.wrap_s;
-      for (int k = 0; k < 4; ++k)
-        if ((rc = make_tmap_window(&al.tm_wrap[k], dqkv, (long long)p.B * p.H, p.W, 3 * p.Ap, p.dp, (k & 1) ? s : e, (k & 2) ? s : e, false)))
-          return rc;
-    }
-    if ((rc = launch_attn_bwd_tc(al, st))) return rc;
-  } else if ((rc = launch_attn_bwd(al, st))) return rc;
+  if ((rc = tc_attn ? launch_attn_bwd_tc(al, st) : launch_attn_bwd(al, st))) return finish(rc);
   // dqkv is complete on the caller's stream: dW_qkv may start on the side stream, next to dx
-  if (ss && (cudaEventRecord(ss->fork2, st) != cudaSuccess || cudaStreamWaitEvent(s2, ss->fork2, 0) != cudaSuccess)) return check_launch();
+  if (ss && (cudaEventRecord(ss->fork2, st) != cudaSuccess || cudaStreamWaitEvent(s2, ss->fork2, 0) != cudaSuccess))
+    return finish(check_launch());
 
   if (dx) {
-    GTLaunch gt{};
-    if ((rc = make_tmap(&gt.tmA, dqkv, p.T, 3 * p.Ap, 128))) return rc;
     gt.natoms = tx.natoms; gt.rows = p.T;
     gt.out = (bf*)dx; gt.ldo = p.C; gt.NB = tx.NB; gt.nstages = tx.nstages; gt.stream_b = tx.stream_b; gt.err = err;
     for (int i = 0; i < tx.nsplit; ++i) {
       const int col0 = i * tx.NB;
       gt.s[i] = GTSplit{bimg + bi.ximg[i], nullptr, col0, (p.C - col0 < tx.NB ? p.C - col0 : tx.NB)};
     }
-    if ((rc = launch_gt(gt, tx.nsplit, st, "dx_gemm"))) return rc;
+    if ((rc = launch_gt(gt, tx.nsplit, st, "dx_gemm"))) return finish(rc);
   }
-  if (dw_qkv || db_qkv) {
+  if (want_dwqkv) {
     // dW_qkv = dqkv^T x (dqkv fetched by TMA); db_qkv from a column of ones appended to x
-    GRLaunch gr{};
-    if ((rc = make_tmap(&gr.tm, dqkv, p.T, 3 * p.Ap, 64))) return rc;
-    gr.tma_is_L = 1;
-    gr.P = (const bf*)x; gr.ldp = p.C; gr.pvalid = p.C;
+    grx.tma_is_L = 1;
+    grx.P = (const bf*)x; grx.ldp = p.C; grx.pvalid = p.C;
     const GrShape gs = gr_shape(p, 1);
-    gr.Ap = p.Ap; gr.dp = p.dp; gr.d = p.d; gr.C = p.C; gr.M = gs.M; gr.rows = p.T;
-    gr.NP = gs.NP; gr.mbpc = gs.mbpc; gr.nsplit = gs.nsplit;
-    gr.out = dw_qkv ? dw_qkv : dummy; gr.colsum = db_qkv; gr.err = err;
-    if ((rc = launch_gr(gr, s2, "dwqkv_gemm"))) return rc;
+    grx.Ap = p.Ap; grx.dp = p.dp; grx.d = p.d; grx.C = p.C; grx.M = gs.M; grx.rows = p.T;
+    grx.NP = gs.NP; grx.mbpc = gs.mbpc; grx.nsplit = gs.nsplit;
+    grx.out = dw_qkv ? dw_qkv : dummy; grx.colsum = db_qkv; grx.err = err;
+    if ((rc = launch_gr(grx, s2, "dwqkv_gemm"))) return finish(rc);
   }
   // the caller's stream continues only after the side stream's work
-  if (ss && (cudaEventRecord(ss->join, s2) != cudaSuccess || cudaStreamWaitEvent(st, ss->join, 0) != cudaSuccess)) return check_launch();
-  return GSWA_OK;
+  return finish(GSWA_OK);
 }
 
 }  // namespace gswa

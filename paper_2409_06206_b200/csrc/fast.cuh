@@ -195,6 +195,12 @@ int launch_attn_bwd(const AttnLaunch& L, cudaStream_t st);
 // Backward on tcgen05 (units of one head only; GSWA_ERR_UNSUPPORTED otherwise).
 int launch_attn_bwd_tc(const AttnLaunch& L, cudaStream_t st);
 
+// Index maps computed by the routines of the tensor-core attention kernels (window 8): win_id[B*H*W] window number
+// b*nW + w of every token in the frame shifted by s, slot[H*W], region[H*W], rel[64*64]; any pointer may be null.
+int launch_fast_index_maps(const FastGeom& g, int s, int32_t* win_id, int32_t* slot, int32_t* region, int32_t* rel,
+                           cudaStream_t st);
+int fast_index_maps(const Plan& p, int group, int32_t* win_id, int32_t* slot, int32_t* region, int32_t* rel, cudaStream_t st);
+
 // ---- orchestration
 bool fast_path_ok(const Plan& p);
 void fast_plan_sizes(Plan* p);

@@ -279,6 +279,37 @@ __global__ void __launch_bounds__(128 * HPU, HPU == 1 ? 4 : 1) attn_bwd_kernel(c
   }
 }
 
+// Index maps as the tensor-core kernels compute them: one block per window of one group runs window_setup (window ->
+// original tokens and mask labels) and the fragment-wise bias-row arithmetic of bias_init, and scatters the results
+// into per-token maps, for a bit-exact comparison with the definition.
+__global__ void __launch_bounds__(128) fast_index_maps_kernel(FastGeom g, int s, int32_t* win_id, int32_t* slot, int32_t* region,
+                                                              int32_t* rel) {
+  __shared__ int tok[64];
+  __shared__ unsigned char reg[64];
+  const int tid = threadIdx.x;
+  window_setup(g, s, (long long)blockIdx.x, tok, reg, tid);
+  __syncthreads();
+  if (tid < 64) {
+    const int token = tok[tid];
+    if (win_id != nullptr) win_id[token] = (int)blockIdx.x;
+    if (blockIdx.x < (unsigned)g.nW) {                       // first image: the per-image maps
+      if (slot != nullptr) slot[token] = tid;
+      if (region != nullptr) region[token] = reg[tid];
+    }
+  }
+  if (rel != nullptr && blockIdx.x == 0) {
+    // the four warps' fragments: thread (warp, lane) holds queries p0 and p0 + 8 against keys 8j + 2t, 8j + 2t + 1
+    const int warp = tid >> 5, lane = tid & 31, p0 = warp * 16 + (lane >> 2), t = lane & 3;
+    for (int j = 0; j < 8; ++j) {
+      const int r = frag_bias_row(p0, t, j), q = 8 * j + 2 * t;
+      rel[p0 * 64 + q] = r;
+      rel[p0 * 64 + q + 1] = r - 1;
+      rel[(p0 + 8) * 64 + q] = r + 15;
+      rel[(p0 + 8) * 64 + q + 1] = r + 14;
+    }
+  }
+}
+
 template <int DP>
 size_t fwd_smem(int nheads) {
   return (size_t)2 * nheads * 3 * 64 * DP * 2 + (size_t)nheads * 225 * 8 + 128 * 4 + 128 + 128 + (size_t)nheads * 4 * 16 * DP * 2;
@@ -341,6 +372,14 @@ int max_heads(const AttnLaunch& L) {
 }
 
 }  // namespace
+
+int launch_fast_index_maps(const FastGeom& g, int s, int32_t* win_id, int32_t* slot, int32_t* region, int32_t* rel,
+                           cudaStream_t st) {
+  if (g.n_windows <= 0) return GSWA_OK;
+  { KernelScope ks_("fast_index_maps", st);
+    fast_index_maps_kernel<<<dim3((unsigned)g.n_windows), 128, 0, st>>>(g, s, win_id, slot, region, rel); }
+  return check_launch();
+}
 
 int launch_attn_fwd(const AttnLaunch& L, cudaStream_t st) {
   const int maxh = max_heads(L);

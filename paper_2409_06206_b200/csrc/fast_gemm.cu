@@ -746,15 +746,7 @@ int launch_prep(const PrepJob* jobs, int njobs, cudaStream_t st, int* err_word) 
   return check_launch();
 }
 
-static int num_sms() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
-  }
-  return n;
-}
+static int num_sms() { return device_sm_count(); }
 
 template <int CP, int DP>
 static int launch_gw_t(const GWLaunch& L, int nunits, cudaStream_t st, const char* name) {

@@ -113,10 +113,13 @@ __global__ void __launch_bounds__(256) colsum_generic(const T* __restrict__ G, l
 }
 
 // ------------------------------------------------------------------------------------------
-// Attention of one (window, head) per block.  qkv is token-major [T,3C] with q already scaled.
+// Attention of one (window, head) per block.  qkv is token-major [T, 2*Cq + Cv] (q | k | v, head-major inside
+// each, q already scaled); q and k have dq columns per head, v and the output dv (Sec. "Parameter Allocation":
+// the Q and K projections may be narrower than V).
 // ------------------------------------------------------------------------------------------
 struct AttnGeom {
-  int H, W, C, nh, d, M, N;
+  int H, W, nh, dq, dv, M, N;
+  int Cq, Cv, ld;              // heads * dq, heads * dv, row length of qkv (2*Cq + Cv)
 };
 
 template <typename T>
@@ -124,11 +127,11 @@ __global__ void __launch_bounds__(128) attn_fwd_generic(AttnGeom g, HeadShifts h
                                                         const T* __restrict__ table, T* __restrict__ A,
                                                         float* __restrict__ L) {
   extern __shared__ float sm[];
-  const int N = g.N, d = g.d, dp = d + 1, Np = N + 1;
+  const int N = g.N, dq = g.dq, dv = g.dv, dqp = dq + 1, dvp = dv + 1, Np = N + 1;
   float* qs = sm;
-  float* ks = qs + N * dp;
-  float* vs = ks + N * dp;
-  float* S = vs + N * dp;
+  float* ks = qs + N * dqp;
+  float* vs = ks + N * dqp;
+  float* S = vs + N * dvp;
   int* tok = reinterpret_cast<int*>(S + N * Np);
   int* reg = tok + N;
   const int h = blockIdx.y, s = hs.s[h];
@@ -142,18 +145,21 @@ __global__ void __launch_bounds__(128) attn_fwd_generic(AttnGeom g, HeadShifts h
     reg[t] = r;
   }
   __syncthreads();
-  for (int e = tid; e < N * d; e += nt) {
-    const int t = e / d, c = e % d;
-    const T* row = qkv + (long long)tok[t] * 3 * g.C + h * d + c;
-    qs[t * dp + c] = ldf(row);
-    ks[t * dp + c] = ldf(row + g.C);
-    vs[t * dp + c] = ldf(row + 2 * g.C);
+  for (int e = tid; e < N * dq; e += nt) {
+    const int t = e / dq, c = e % dq;
+    const T* row = qkv + (long long)tok[t] * g.ld + h * dq + c;
+    qs[t * dqp + c] = ldf(row);
+    ks[t * dqp + c] = ldf(row + g.Cq);
+  }
+  for (int e = tid; e < N * dv; e += nt) {
+    const int t = e / dv, c = e % dv;
+    vs[t * dvp + c] = ldf(qkv + (long long)tok[t] * g.ld + 2 * g.Cq + h * dv + c);
   }
   __syncthreads();
   for (int e = tid; e < N * N; e += nt) {
     const int p = e / N, q = e % N;
     float acc = 0.f;
-    for (int c = 0; c < d; ++c) acc = fmaf(qs[p * dp + c], ks[q * dp + c], acc);
+    for (int c = 0; c < dq; ++c) acc = fmaf(qs[p * dqp + c], ks[q * dqp + c], acc);
     acc += ldf(table + rel_row(g.M, p, q) * g.nh + h);
     S[p * Np + q] = (reg[p] == reg[q]) ? acc : -INFINITY;
   }
@@ -175,15 +181,17 @@ __global__ void __launch_bounds__(128) attn_fwd_generic(AttnGeom g, HeadShifts h
     if (lane == 0 && L != nullptr) L[(long long)tok[p] * g.nh + h] = mx + logf(sum);
   }
   __syncthreads();
-  for (int e = tid; e < N * d; e += nt) {
-    const int p = e / d, c = e % d;
+  for (int e = tid; e < N * dv; e += nt) {
+    const int p = e / dv, c = e % dv;
     float acc = 0.f;
-    for (int q = 0; q < N; ++q) acc = fmaf(S[p * Np + q], vs[q * dp + c], acc);
-    stf(A + (long long)tok[p] * g.C + h * d + c, acc);
+    for (int q = 0; q < N; ++q) acc = fmaf(S[p * Np + q], vs[q * dvp + c], acc);
+    stf(A + (long long)tok[p] * g.Cv + h * dv + c, acc);
   }
 }
 
-// Backward of one (window, head): recompute P from q, k and the saved row log-sum-exp.
+// Backward of one (window, head): recompute P from q, k and the saved row log-sum-exp.  One N x N buffer serves
+// two passes (first P, for dV = P^T dO; then, in place, dS = P o (dP - D), for dQ and dK), so that a 12 x 12
+// window with head dims up to 48 fits the shared memory of one block.
 template <typename T>
 __global__ void __launch_bounds__(256) attn_bwd_generic(AttnGeom g, HeadShifts hs, float scale,
                                                         const T* __restrict__ qkv, const T* __restrict__ table,
@@ -191,14 +199,13 @@ __global__ void __launch_bounds__(256) attn_bwd_generic(AttnGeom g, HeadShifts h
                                                         const T* __restrict__ dA, T* __restrict__ dqkv,
                                                         float* __restrict__ dtable) {
   extern __shared__ float sm[];
-  const int N = g.N, d = g.d, dp = d + 1, Np = N + 1, nrel = (2 * g.M - 1) * (2 * g.M - 1);
+  const int N = g.N, dq = g.dq, dv = g.dv, dqp = dq + 1, dvp = dv + 1, Np = N + 1, nrel = (2 * g.M - 1) * (2 * g.M - 1);
   float* qs = sm;
-  float* ks = qs + N * dp;
-  float* vs = ks + N * dp;
-  float* dOs = vs + N * dp;
-  float* P = dOs + N * dp;
-  float* dS = P + N * Np;
-  float* D = dS + N * Np;
+  float* ks = qs + N * dqp;
+  float* vs = ks + N * dqp;
+  float* dOs = vs + N * dvp;
+  float* PS = dOs + N * dvp;                // P, then dS
+  float* D = PS + N * Np;
   float* Ls = D + N;
   float* hist = Ls + N;
   int* tok = reinterpret_cast<int*>(hist + nrel);
@@ -216,50 +223,61 @@ __global__ void __launch_bounds__(256) attn_bwd_generic(AttnGeom g, HeadShifts h
   }
   for (int e = tid; e < nrel; e += nt) hist[e] = 0.f;
   __syncthreads();
-  for (int e = tid; e < N * d; e += nt) {
-    const int t = e / d, c = e % d;
-    const T* row = qkv + (long long)tok[t] * 3 * g.C + h * d + c;
-    qs[t * dp + c] = ldf(row);
-    ks[t * dp + c] = ldf(row + g.C);
-    vs[t * dp + c] = ldf(row + 2 * g.C);
-    dOs[t * dp + c] = ldf(dA + (long long)tok[t] * g.C + h * d + c);
+  for (int e = tid; e < N * dq; e += nt) {
+    const int t = e / dq, c = e % dq;
+    const T* row = qkv + (long long)tok[t] * g.ld + h * dq + c;
+    qs[t * dqp + c] = ldf(row);
+    ks[t * dqp + c] = ldf(row + g.Cq);
+  }
+  for (int e = tid; e < N * dv; e += nt) {
+    const int t = e / dv, c = e % dv;
+    vs[t * dvp + c] = ldf(qkv + (long long)tok[t] * g.ld + 2 * g.Cq + h * dv + c);
+    dOs[t * dvp + c] = ldf(dA + (long long)tok[t] * g.Cv + h * dv + c);
   }
   __syncthreads();
   // D_p = sum_c dO[p,c] O[p,c]
   for (int p = tid; p < N; p += nt) {
     float acc = 0.f;
-    for (int c = 0; c < d; ++c) acc = fmaf(dOs[p * dp + c], ldf(A + (long long)tok[p] * g.C + h * d + c), acc);
+    for (int c = 0; c < dv; ++c) acc = fmaf(dOs[p * dvp + c], ldf(A + (long long)tok[p] * g.Cv + h * dv + c), acc);
     D[p] = acc;
   }
-  __syncthreads();
+  // pass 1: P
   for (int e = tid; e < N * N; e += nt) {
     const int p = e / N, q = e % N;
-    float sc = 0.f, dpv = 0.f;
-    for (int c = 0; c < d; ++c) {
-      sc = fmaf(qs[p * dp + c], ks[q * dp + c], sc);
-      dpv = fmaf(dOs[p * dp + c], vs[q * dp + c], dpv);
-    }
-    const int rr = rel_row(g.M, p, q);
-    sc += ldf(table + rr * g.nh + h);
-    const float pv = (reg[p] == reg[q]) ? expf(sc - Ls[p]) : 0.f;
-    const float ds = pv * (dpv - D[p]);
-    P[p * Np + q] = pv;
-    dS[p * Np + q] = ds;
-    if (dtable != nullptr && pv != 0.f) atomicAdd(hist + rr, ds);
+    float sc = 0.f;
+    for (int c = 0; c < dq; ++c) sc = fmaf(qs[p * dqp + c], ks[q * dqp + c], sc);
+    sc += ldf(table + rel_row(g.M, p, q) * g.nh + h);
+    PS[p * Np + q] = (reg[p] == reg[q]) ? expf(sc - Ls[p]) : 0.f;
   }
   __syncthreads();
-  for (int e = tid; e < N * d; e += nt) {
-    const int t = e / d, c = e % d;
-    float aq = 0.f, ak = 0.f, av = 0.f;
+  for (int e = tid; e < N * dv; e += nt) {
+    const int t = e / dv, c = e % dv;
+    float av = 0.f;
+    for (int u = 0; u < N; ++u) av = fmaf(PS[u * Np + t], dOs[u * dvp + c], av);
+    stf(dqkv + (long long)tok[t] * g.ld + 2 * g.Cq + h * dv + c, av);
+  }
+  __syncthreads();
+  // pass 2: dS in place
+  for (int e = tid; e < N * N; e += nt) {
+    const int p = e / N, q = e % N;
+    const float pv = PS[p * Np + q];
+    float dpv = 0.f;
+    for (int c = 0; c < dv; ++c) dpv = fmaf(dOs[p * dvp + c], vs[q * dvp + c], dpv);
+    const float ds = pv * (dpv - D[p]);
+    PS[p * Np + q] = ds;
+    if (dtable != nullptr && pv != 0.f) atomicAdd(hist + rel_row(g.M, p, q), ds);
+  }
+  __syncthreads();
+  for (int e = tid; e < N * dq; e += nt) {
+    const int t = e / dq, c = e % dq;
+    float aq = 0.f, ak = 0.f;
     for (int u = 0; u < N; ++u) {
-      aq = fmaf(dS[t * Np + u], ks[u * dp + c], aq);
-      ak = fmaf(dS[u * Np + t], qs[u * dp + c], ak);
-      av = fmaf(P[u * Np + t], dOs[u * dp + c], av);
+      aq = fmaf(PS[t * Np + u], ks[u * dqp + c], aq);
+      ak = fmaf(PS[u * Np + t], qs[u * dqp + c], ak);
     }
-    T* row = dqkv + (long long)tok[t] * 3 * g.C + h * d + c;
+    T* row = dqkv + (long long)tok[t] * g.ld + h * dq + c;
     stf(row, aq * scale);
-    stf(row + g.C, ak);
-    stf(row + 2 * g.C, av);
+    stf(row + g.Cq, ak);
   }
   if (dtable != nullptr)
     for (int e = tid; e < nrel; e += nt) atomicAdd(dtable + e * g.nh + h, hist[e]);
@@ -327,10 +345,8 @@ HeadShifts head_shifts(const Plan& p) {
   return hs;
 }
 
-size_t attn_fwd_smem(const Plan& p) { return sizeof(float) * (3 * p.N * (p.d + 1) + p.N * (p.N + 1)) + 8 * p.N; }
-size_t attn_bwd_smem(const Plan& p) {
-  const int nrel = (2 * p.M - 1) * (2 * p.M - 1);
-  return sizeof(float) * (4 * p.N * (p.d + 1) + 2 * p.N * (p.N + 1) + 2 * p.N + nrel) + 8 * p.N;
+AttnGeom attn_geom(const Plan& p) {
+  return AttnGeom{p.H, p.W, p.nh, p.dqk, p.dv, p.M, p.N, p.Cq, p.Cv, p.Cqkv};
 }
 
 template <typename T>
@@ -340,16 +356,15 @@ int forward_t(const Plan& p, const T* x, const T* w_qkv, const T* b_qkv, const T
   T* A = reinterpret_cast<T*>(saved + p.off_A);
   float* L = reinterpret_cast<float*>(saved + p.off_L);
   const int C = p.C;
-  const float scale = 1.0f / sqrtf((float)p.d);
-  int rc = launch_gemm<T, T, T>(x, C, 1, w_qkv, 1, C, qkv, 3 * C, b_qkv, p.T, 3 * C, C, scale, C, st);
-  if (rc) return rc;
-  AttnGeom g{p.H, p.W, C, p.nh, p.d, p.M, p.N};
-  const size_t smem = attn_fwd_smem(p);
+  const float scale = 1.0f / sqrtf((float)p.dqk);
+  const size_t smem = generic_attn_fwd_smem(p);
   if (cudaFuncSetAttribute(attn_fwd_generic<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return check_launch();
-  { KernelScope ks_("attn_fwd_generic", st); attn_fwd_generic<T><<<dim3(p.B * p.nW, p.nh), 128, smem, st>>>(g, head_shifts(p), qkv, table, A, L); }
+  int rc = launch_gemm<T, T, T>(x, C, 1, w_qkv, 1, C, qkv, p.Cqkv, b_qkv, p.T, p.Cqkv, C, scale, p.Cq, st);
+  if (rc) return rc;
+  { KernelScope ks_("attn_fwd_generic", st); attn_fwd_generic<T><<<dim3(p.B * p.nW, p.nh), 128, smem, st>>>(attn_geom(p), head_shifts(p), qkv, table, A, L); }
   if ((rc = check_launch())) return rc;
-  return launch_gemm<T, T, T>(A, C, 1, w_proj, 1, C, y, C, b_proj, p.T, C, C, 1.f, 0, st);
+  return launch_gemm<T, T, T>(A, p.Cv, 1, w_proj, 1, p.Cv, y, C, b_proj, p.T, C, p.Cv, 1.f, 0, st);
 }
 
 template <typename T>
@@ -359,30 +374,39 @@ int backward_t(const Plan& p, const T* x, const T* w_qkv, const T* w_proj, const
   const T* qkv = reinterpret_cast<const T*>(saved + p.off_qkv);
   const T* A = reinterpret_cast<const T*>(saved + p.off_A);
   const float* L = reinterpret_cast<const float*>(saved + p.off_L);
-  const int C = p.C;
+  const int C = p.C, Cv = p.Cv, Q = p.Cqkv;
   T* dA = reinterpret_cast<T*>(scratch);
-  T* dqkv = dA + p.T * C;
-  const float scale = 1.0f / sqrtf((float)p.d);
+  T* dqkv = dA + p.T * Cv;
+  const float scale = 1.0f / sqrtf((float)p.dqk);
   int rc;
-  // dA = dy W_proj
-  if ((rc = launch_gemm<T, T, T>(dy, C, 1, w_proj, C, 1, dA, C, nullptr, p.T, C, C, 1.f, 0, st))) return rc;
-  if (dw_proj && (rc = launch_gemm_tn<T, T>(dy, C, C, A, C, C, p.T, dw_proj, st))) return rc;
-  if (db_proj && (rc = launch_colsum<T>(dy, p.T, C, C, db_proj, st))) return rc;
-  AttnGeom g{p.H, p.W, C, p.nh, p.d, p.M, p.N};
-  const size_t smem = attn_bwd_smem(p);
+  // every fallible host-side step comes before the first launch
+  const size_t smem = generic_attn_bwd_smem(p);
   if (cudaFuncSetAttribute(attn_bwd_generic<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return check_launch();
-  { KernelScope ks_("attn_bwd_generic", st); attn_bwd_generic<T><<<dim3(p.B * p.nW, p.nh), 256, smem, st>>>(g, head_shifts(p), scale, qkv, table, A, L, dA, dqkv,
+  // dA = dy W_proj
+  if ((rc = launch_gemm<T, T, T>(dy, C, 1, w_proj, Cv, 1, dA, Cv, nullptr, p.T, Cv, C, 1.f, 0, st))) return rc;
+  if (dw_proj && (rc = launch_gemm_tn<T, T>(dy, C, C, A, Cv, Cv, p.T, dw_proj, st))) return rc;
+  if (db_proj && (rc = launch_colsum<T>(dy, p.T, C, C, db_proj, st))) return rc;
+  { KernelScope ks_("attn_bwd_generic", st); attn_bwd_generic<T><<<dim3(p.B * p.nW, p.nh), 256, smem, st>>>(attn_geom(p), head_shifts(p), scale, qkv, table, A, L, dA, dqkv,
                                                                  dtable); }
   if ((rc = check_launch())) return rc;
-  if (dx && (rc = launch_gemm<T, T, T>(dqkv, 3 * C, 1, w_qkv, C, 1, dx, C, nullptr, p.T, C, 3 * C, 1.f, 0, st)))
+  if (dx && (rc = launch_gemm<T, T, T>(dqkv, Q, 1, w_qkv, C, 1, dx, C, nullptr, p.T, C, Q, 1.f, 0, st)))
     return rc;
-  if (dw_qkv && (rc = launch_gemm_tn<T, T>(dqkv, 3 * C, 3 * C, x, C, C, p.T, dw_qkv, st))) return rc;
-  if (db_qkv && (rc = launch_colsum<T>(dqkv, p.T, 3 * C, 3 * C, db_qkv, st))) return rc;
+  if (dw_qkv && (rc = launch_gemm_tn<T, T>(dqkv, Q, Q, x, C, C, p.T, dw_qkv, st))) return rc;
+  if (db_qkv && (rc = launch_colsum<T>(dqkv, p.T, Q, Q, db_qkv, st))) return rc;
   return GSWA_OK;
 }
 
 }  // namespace
+
+size_t generic_attn_fwd_smem(const Plan& p) {
+  return sizeof(float) * ((size_t)2 * p.N * (p.dqk + 1) + (size_t)p.N * (p.dv + 1) + (size_t)p.N * (p.N + 1)) + 8 * (size_t)p.N;
+}
+size_t generic_attn_bwd_smem(const Plan& p) {
+  const size_t nrel = (size_t)(2 * p.M - 1) * (2 * p.M - 1);
+  return sizeof(float) * ((size_t)2 * p.N * (p.dqk + 1) + (size_t)2 * p.N * (p.dv + 1) + (size_t)p.N * (p.N + 1) + 2 * p.N + nrel) +
+         8 * (size_t)p.N;
+}
 
 int generic_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
                     const void* b_proj, const void* table, void* y, void* saved, cudaStream_t st) {
@@ -429,6 +453,48 @@ int launch_zero(float* const* ptrs, const long long* counts, int nbuf, cudaStrea
 
 int launch_colsum_bf16(const __nv_bfloat16* G, long long rows, int cols, long long ld, float* out, cudaStream_t st) {
   return launch_colsum<__nv_bfloat16>(G, rows, cols, ld, out, st);
+}
+
+__global__ void batch_window_ids_kernel(int B, int H, int W, int M, int s, int32_t* win_id) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (long long)B * H * W) return;
+  const int b = (int)(idx / (H * W)), rem = (int)(idx % (H * W));
+  int w, t, r;
+  token_to_slot(H, W, M, s, rem / W, rem % W, &w, &t, &r);
+  win_id[idx] = b * (H / M) * (W / M) + w;
+}
+
+int launch_batch_window_ids(const Plan& p, int group, int32_t* win_id, cudaStream_t st) {
+  if (p.T == 0) return GSWA_OK;
+  { KernelScope ks_("batch_window_ids", st);
+    batch_window_ids_kernel<<<(unsigned)((p.T + 255) / 256), 256, 0, st>>>(p.B, p.H, p.W, p.M, p.gs[group], win_id); }
+  return check_launch();
+}
+
+// The give-up path of a bounded wait, on purpose: a barrier that expects one arrival and never gets it.  The poll
+// limit is small, the kernel returns normally, and the only trace is the error word.
+__global__ void wait_timeout_kernel(int* err) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"((uint32_t)__cvta_generic_to_shared(&bar)) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    bool done = false;
+    for (int i = 0; i < 2000 && !done; ++i) {
+      uint32_t ok;
+      asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], 0;\n\tselp.b32 %0, 1, 0, p;\n\t}\n"
+                   : "=r"(ok)
+                   : "r"((uint32_t)__cvta_generic_to_shared(&bar))
+                   : "memory");
+      done = ok != 0;
+      if (!done) __nanosleep(32);
+    }
+    if (!done) atomicExch(err, 1);
+  }
+}
+
+int launch_wait_timeout(int* err, cudaStream_t st) {
+  { KernelScope ks_("wait_timeout", st); wait_timeout_kernel<<<1, 32, 0, st>>>(err); }
+  return check_launch();
 }
 
 int launch_index_maps(const Plan& p, int group, int32_t* win, int32_t* slot, int32_t* region, int32_t* token_of,

@@ -16,6 +16,8 @@ constexpr int kMaxHeads = 64;
 // Validated, flattened copy of a gswa_desc plus derived sizes.
 struct Plan {
   int B, H, W, C, nh, d, M, N, G;
+  int dqk, dv;                 // per-head widths of q,k and of v (d unless the descriptor narrows them)
+  int Cq, Cv, Cqkv;            // heads*dqk, heads*dv, 2*Cq + Cv (rows of w_qkv)
   int nWh, nWw, nW;            // windows per image: rows, cols, total
   long long T;                 // tokens = B*H*W
   int dtype;
@@ -40,6 +42,7 @@ struct HeadShifts {
 int make_plan(const gswa_desc* desc, Plan* plan);
 int check_launch();  // GSWA_OK or GSWA_ERR_CUDA (records the CUDA error text)
 int launch_zero(float* const* ptrs, const long long* counts, int nbuf, cudaStream_t st);   // one launch zeroes them all
+int device_sm_count();     // multiprocessors of the current device (148 if the query fails)
 bool profiling_enabled();  // per-kernel event timing is on (kernels are then kept on one stream)
 
 // Wraps one kernel launch: counts it and, while profiling is enabled, brackets it with a CUDA
@@ -57,8 +60,15 @@ int generic_forward(const Plan& p, const void* x, const void* w_qkv, const void*
 int generic_backward(const Plan& p, const void* x, const void* w_qkv, const void* w_proj, const void* table,
                      const void* saved, const void* dy, void* dx, float* dw_qkv, float* db_qkv, float* dw_proj,
                      float* db_proj, float* dtable, void* scratch, cudaStream_t st);
+size_t generic_attn_fwd_smem(const Plan& p);   // dynamic shared memory of the generic attention kernels
+size_t generic_attn_bwd_smem(const Plan& p);
 int launch_colsum_bf16(const __nv_bfloat16* G, long long rows, int cols, long long ld, float* out, cudaStream_t st);
 int launch_index_maps(const Plan& p, int group, int32_t* win, int32_t* slot, int32_t* region, int32_t* token_of,
                       int32_t* rel, cudaStream_t st);
+// win_id[B*H*W] = b*nW + window of every token (the per-image map of launch_index_maps repeated over the batch)
+int launch_batch_window_ids(const Plan& p, int group, int32_t* win_id, cudaStream_t st);
+// A one-block kernel that waits on a barrier nobody arrives on, gives up after a few thousand polls and sets the
+// device error word at `err` (the path every bounded wait of the tensor-core kernels takes when it runs out).
+int launch_wait_timeout(int* err, cudaStream_t st);
 
 }  // namespace gswa

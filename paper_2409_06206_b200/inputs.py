@@ -8,7 +8,9 @@ Recipe (stands in for the paper's DIV2K training patches and test images,
 Sec. "Experimental Setup"): activations entering the attention layer follow a
 LayerNorm (Eq. 4), hence x ~ N(0,1); projection weights and the
 relative-position bias table ~ N(0, 0.02^2); projection biases zero unless a
-test asks otherwise; upstream gradient dy ~ N(0,1).  For bf16 workloads every
+test asks otherwise; upstream gradient dy ~ N(0,1).  Tests that must excite
+the attention scores (a softmax far from uniform) raise the weight and table
+standard deviations through `w_std` / `table_std`.  For bf16 workloads every
 sample is rounded to the nearest bf16 value (ties to even) before anybody sees
 it, and returned as float32 holding exactly that value.
 """
@@ -38,6 +40,10 @@ class LayerConfig:
     layers: int = 1                  # stacked-inference workloads call the layer this many times
     backward: bool = True
     bias_std: float = 0.0            # std of b_qkv / b_proj (0 in the paper-shaped workloads)
+    w_std: float = 0.02              # std of w_qkv / w_proj
+    table_std: float = 0.02          # std of the relative-position bias table
+    qk_dim: int = 0                  # per-head width of Q and K (0 = head dim; Sec. "Parameter Allocation")
+    v_dim: int = 0                   # per-head width of V (0 = head dim)
 
     @property
     def tokens(self) -> int:
@@ -46,6 +52,17 @@ class LayerConfig:
     @property
     def head_dim(self) -> int:
         return self.C // self.num_heads
+
+    @property
+    def qkv_rows(self) -> int:
+        """Rows of w_qkv: heads * (2 * qk width + v width); 3C by default."""
+        d = self.head_dim
+        return self.num_heads * (2 * (self.qk_dim or d) + (self.v_dim or d))
+
+    @property
+    def v_cols(self) -> int:
+        """Columns of w_proj: heads * v width; C by default."""
+        return self.num_heads * (self.v_dim or self.head_dim)
 
 
 # The workloads the layer is measured and checked on.  Batch 16..256 and C=60
@@ -104,11 +121,11 @@ def make_inputs(cfg: LayerConfig, layer: int = 0, batch: int | None = None,
     C, M, nh = cfg.C, cfg.window, cfg.num_heads
     shapes = {
         "x": ((B, cfg.H, cfg.W, C), 1.0),
-        "w_qkv": ((3 * C, C), 0.02),
-        "b_qkv": ((3 * C,), cfg.bias_std),
-        "w_proj": ((C, C), 0.02),
+        "w_qkv": ((cfg.qkv_rows, C), cfg.w_std),
+        "b_qkv": ((cfg.qkv_rows,), cfg.bias_std),
+        "w_proj": ((C, cfg.v_cols), cfg.w_std),
         "b_proj": ((C,), cfg.bias_std),
-        "bias_table": (((2 * M - 1) ** 2, nh), 0.02),
+        "bias_table": (((2 * M - 1) ** 2, nh), cfg.table_std),
         "dy": ((B, cfg.H, cfg.W, C), 1.0),
     }
     out = {}

@@ -40,9 +40,15 @@ def test_workspace_query_and_descriptor_validation():
         (gb.Desc(1, 16, 16, 60, 6, 8, (3, 2), (0, 4)), -2),       # heads do not add up
         (gb.Desc(1, 16, 16, 60, 6, 8, (3, 3), (0, 8)), -2),       # shift out of range
         (gb.Desc(1, 16, 16, 62, 6, 8, (3, 3), (0, 4)), -2),       # C not divisible by heads
-        (gb.Desc(1, 16, 16, 60, 6, 8, (3, 3), (0, 4), qk_dim=16), -4),
+        (gb.Desc(1, 16, 16, 60, 6, 8, (3, 3), (0, 4), qk_dim=65), -4),     # wider than the kernels' head-dim limit
+        (gb.Desc(1, 24, 24, 128, 2, 12, (1, 1), (0, 6), "f32"), -4),        # a 12 x 12 window with head dim 64: more shared memory than a block has
         (gb.Desc(1, 16, 16, 60, 6, 8, (), ()), -2),
     ]
+    # narrowed Q/K projections (Sec. "Parameter Allocation") and the paper's window 12 are accepted
+    narrow = gb.Desc(2, 24, 24, 180, 6, 12, (3, 3), (0, 6), "bf16", qk_dim=16)
+    wide = gb.Desc(2, 24, 24, 180, 6, 12, (3, 3), (0, 6), "bf16")
+    assert gb.gswa_workspace_query(narrow)[0] < gb.gswa_workspace_query(wide)[0]
+    assert gb.gswa_workspace_query(gb.Desc(1, 24, 24, 180, 6, 12, (3, 3), (0, 6), "bf16"))[3] > 0   # window 12, head dim 30
     for desc, code in bad:
         with pytest.raises(gb.GswaError) as e:
             gb.gswa_workspace_query(desc)

@@ -11,7 +11,7 @@ from paper_2409_06206_b200 import binding as gb
 from paper_2409_06206_b200 import build as gbuild
 from paper_2409_06206_b200.inputs import CONFIGS, LayerConfig, make_inputs
 
-from gpu_util import GRADS, assert_close, rel_err, run_gpu, run_oracle
+from gpu_util import EXCITED, GRADS, assert_close, rel_err, run_gpu, run_oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -42,6 +42,52 @@ def test_index_maps_bit_exact(H, W, M, s):
     assert np.array_equal(rel.cpu().numpy(), rel_ref.ravel())
 
 
+@pytest.mark.parametrize("B,H,W,s,dtype,C,nh", [(2, 16, 16, 4, "bf16", 64, 2), (3, 16, 24, 3, "bf16", 180, 6), (1, 64, 64, 4, "bf16", 60, 6),
+                                               (2, 8, 8, 7, "bf16", 64, 4), (1, 8, 16, 1, "bf16", 96, 6), (2, 24, 12, 1, "f32", 12, 2)])
+def test_debug_index_maps_of_the_running_path_bit_exact(B, H, W, s, dtype, C, nh):
+    """The maps as the kernels that run the layer compute them (on the bf16 path: the window set-up and the
+    fragment-wise bias rows of the tensor-core attention kernels), over the whole batch, bit for bit."""
+    import torch
+    M = 8 if dtype == "bf16" else 4
+    d = gb.Desc(B, H, W, C, nh, M, (nh - 1, 1), (0, s), dtype)
+    N, nW = M * M, (H // M) * (W // M)
+    win_id = torch.full((B * H * W,), -1, dtype=torch.int32, device="cuda")
+    slot = torch.full((H * W,), -1, dtype=torch.int32, device="cuda")
+    region = torch.full((H * W,), -1, dtype=torch.int32, device="cuda")
+    rel = torch.full((N * N,), -1, dtype=torch.int32, device="cuda")
+    gb.gswa_debug_index_maps(d, 1, win_id, slot, region, rel)
+    torch.cuda.synchronize()
+    win, slot_ref, region_ref, rel_ref = orc.index_maps(H, W, M, s)
+    want = (np.arange(B, dtype=np.int32)[:, None] * nW + win.ravel()[None, :]).ravel()
+    assert np.array_equal(win_id.cpu().numpy(), want)
+    assert np.array_equal(slot.cpu().numpy(), slot_ref.ravel())
+    assert np.array_equal(region.cpu().numpy(), region_ref.ravel())
+    assert np.array_equal(rel.cpu().numpy(), rel_ref.ravel())
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_harmless():
+    """A device-side wait expires on purpose (a barrier nobody arrives on, about two thousand polls): the error word
+    is set, gswa_scratch_status reports GSWA_ERR_DEVICE, and the next call on the same scratch is correct."""
+    import torch
+    cfg = SWEEP[8]
+    inp = make_inputs(cfg)
+    desc = gb.Desc.from_config(cfg)
+    scratch = torch.zeros(max(gb.gswa_workspace_query(desc)[1:]), dtype=torch.uint8, device="cuda")
+    gb.gswa_scratch_status(desc, scratch)                       # clean
+    gb.gswa_debug_expire_wait(desc, scratch)
+    with pytest.raises(gb.GswaError) as e:
+        gb.gswa_scratch_status(desc, scratch)
+    assert e.value.status == -7
+    torch.cuda.synchronize()
+    got = run_gpu(cfg, inp)                                     # the context is intact
+    assert_close(got, run_oracle(cfg, inp), cfg.dtype)
+    # a forward call on the same scratch clears the word
+    dev = {k: __import__("gpu_util").to_device(v, cfg.dtype) for k, v in inp.items()}
+    y = torch.empty(inp["x"].shape, dtype=torch.bfloat16, device="cuda")
+    gb.gswa_forward(desc, dev["x"], dev["w_qkv"], dev["b_qkv"], dev["w_proj"], dev["b_proj"], dev["bias_table"], y, None, scratch)
+    gb.gswa_scratch_status(desc, scratch)
+
+
 def test_config1_f32_forward_backward():
     cfg = CONFIGS["c1"]
     inp = make_inputs(cfg)
@@ -69,7 +115,33 @@ SWEEP = [
     _mk("s10", 3, 24, 40, 60, 6, 8, (6,), (4,), "bf16"),
     _mk("s11", 5, 16, 16, 64, 2, 8, (1, 1), (0, 1), "bf16"),
     _mk("s12", 1, 24, 24, 36, 3, 12, (1, 2), (0, 6), "bf16"),
+    # more heads than the attention kernels have one-head work units for: their multi-head CTAs run
+    _mk("s13", 2, 16, 24, 192, 12, 8, (6, 6), (0, 4), "bf16"),
+    _mk("s14", 1, 24, 16, 180, 10, 8, (5, 5), (3, 0), "bf16"),
+    _mk("s15", 2, 16, 16, 240, 12, 8, (4, 8), (4, 1), "bf16"),
 ]
+
+
+# The paper's own layer settings (Sec. "Parameter Allocation", Sec. "Experimental Setup"): Q and K narrowed to 16
+# channels (read per head, and read as the total over heads), window 12; plus the window-12 layer at C = 180 whose
+# backward needs the most shared memory of all supported shapes.
+PAPER_SHAPES = [
+    dataclasses.replace(_mk("p0", 2, 24, 24, 180, 6, 12, (3, 3), (0, 6), "f32"), qk_dim=16),
+    dataclasses.replace(_mk("p1", 2, 24, 24, 180, 6, 12, (3, 3), (0, 6), "bf16"), qk_dim=16),
+    dataclasses.replace(_mk("p2", 2, 24, 36, 60, 4, 12, (2, 2), (6, 0), "f32"), qk_dim=4),
+    dataclasses.replace(_mk("p3", 2, 24, 36, 60, 4, 12, (2, 2), (6, 0), "bf16"), qk_dim=4),
+    dataclasses.replace(_mk("p4", 1, 16, 16, 60, 6, 8, (3, 3), (0, 4), "bf16"), qk_dim=16, v_dim=12),
+    _mk("p5", 1, 24, 24, 180, 6, 12, (3, 3), (0, 6), "f32"),
+    _mk("p6", 1, 24, 24, 180, 6, 12, (3, 3), (0, 6), "bf16"),
+]
+
+
+@pytest.mark.parametrize("cfg", PAPER_SHAPES, ids=[c.name for c in PAPER_SHAPES])
+def test_narrowed_qk_projections_and_window_12(cfg):
+    inp = make_inputs(cfg)
+    got = run_gpu(cfg, inp)
+    ref = run_oracle(cfg, inp)
+    assert_close(got, ref, cfg.dtype)
 
 
 @pytest.mark.parametrize("cfg", SWEEP, ids=[c.name for c in SWEEP])
@@ -112,6 +184,20 @@ def test_random_shapes_tensor_core_path(cfg):
     assert_close(run_gpu(cfg, inp), ref, cfg.dtype)
     assert_close(run_gpu(cfg, inp, flags=gb.FLAG_FUSED_FWD), ref, cfg.dtype)
     assert_close(run_gpu(cfg, inp, flags=gb.FLAG_TCGEN05_ATTN), ref, cfg.dtype)
+
+
+@pytest.mark.parametrize("flags", [0, gb.FLAG_FUSED_FWD, gb.FLAG_TCGEN05_ATTN, gb.FLAG_GENERIC],
+                         ids=["default", "fused-fwd", "tcgen05-attn", "generic"])
+@pytest.mark.parametrize("cfg", EXCITED, ids=[c.name for c in EXCITED])
+def test_score_exciting_inputs(cfg, flags):
+    """Weights ~ N(0, 1/C) and a table of std 0.7: the softmax is far from uniform, so the bias gather, the query
+    scale and the mask all move y and the gradients well beyond the tolerance if they are wrong
+    (tests/test_parity_inputs_bite.py proves that on the CPU).  The q / k / v row blocks of dw_qkv and db_qkv are
+    measured separately, each against its own largest entry."""
+    inp = make_inputs(cfg)
+    ref = run_oracle(cfg, inp)
+    errs = assert_close(run_gpu(cfg, inp, flags=flags), ref, cfg.dtype, blocks_of=cfg.C)
+    assert {"dw_qkv_q", "dw_qkv_k", "dw_qkv_v", "db_qkv_q", "db_qkv_v"} <= set(errs)
 
 
 @pytest.mark.parametrize("cfg", [SWEEP[2], SWEEP[7], SWEEP[8]], ids=["f32", "bf16-c60", "bf16-c180"])
@@ -189,24 +275,32 @@ def test_training_shapes_reduced_batch(name, batch):
 
 
 @pytest.mark.parametrize("name", ["cM", "c4"])
-def test_full_size_sampled_images_and_properties(name):
-    """Full-size launch configuration: y and dx of sampled batch items against the checker (batch items are
-    independent), plus properties of the parameter gradients that hold at any size."""
+def test_full_size_every_tensor_against_the_checker(name):
+    """Full-size launch configuration, the one bench.py times: all seven result tensors against the checker, which
+    walks the whole batch a few images at a time (y and dx are compared chunk by chunk, the parameter gradients
+    are summed over all chunks and compared at the end).  The weight-gradient GEMMs wrap their operand rings
+    dozens of times only at this size."""
     cfg = CONFIGS[name]
     inp = make_inputs(cfg)
-    got = run_gpu(cfg, inp)
-    picks = [0, cfg.B // 2 + 1, cfg.B - 1]
-    sub = {k: (v[picks] if k in ("x", "dy") else v) for k, v in inp.items()}
-    ref = run_oracle(cfg, sub, chunk=3)
-    assert rel_err(got["y"][picks], ref["y"]) <= 2e-2
-    assert rel_err(got["dx"][picks], ref["dx"]) <= 2e-2
-    dy2 = inp["dy"].reshape(-1, cfg.C).astype(np.float64)
-    assert rel_err(got["db_proj"], dy2.sum(0)) <= 2e-2
-    scale = np.abs(got["dbias_table"]).max()
-    assert np.abs(got["dbias_table"].sum(0)).max() <= 2e-2 * scale * 15       # columns sum to 0 (softmax invariance)
-    assert np.abs(got["db_qkv"][cfg.C:2 * cfg.C]).max() <= 2e-2 * np.abs(got["db_qkv"]).max()   # key bias gradient is 0
-    for n in GRADS:
-        assert np.isfinite(got[n]).all()
+    got = run_gpu(cfg, inp, as_float32=True)
+    gh, gs = cfg.group_heads, cfg.group_shift
+    chunk, acc = 4, None
+    num = {"y": 0.0, "dx": 0.0}
+    den = {"y": 0.0, "dx": 0.0}
+    for b0 in range(0, cfg.B, chunk):
+        sl = slice(b0, b0 + chunk)
+        y, cache = orc.forward(inp["x"][sl], inp["w_qkv"], inp["b_qkv"], inp["w_proj"], inp["b_proj"], inp["bias_table"],
+                               cfg.window, gh, gs)
+        g = orc.backward(cache, inp["dy"][sl])
+        for n, r in (("y", y), ("dx", g.pop("dx"))):
+            num[n] = max(num[n], float(np.abs(got[n][sl] - r).max()))
+            den[n] = max(den[n], float(np.abs(r).max()))
+        acc = g if acc is None else {n: acc[n] + g[n] for n in acc}
+    errs = {n: num[n] / den[n] for n in num}
+    errs.update({n: rel_err(got[n].astype(np.float64), acc[n]) for n in acc})
+    bad = {n: e for n, e in errs.items() if not e <= 2e-2}
+    assert not bad, "beyond 2e-2: %s (all: %s)" % (bad, errs)
+    assert set(errs) == set(GRADS) | {"y"}
 
 
 def test_stacked_inference_layers():

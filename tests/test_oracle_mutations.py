@@ -26,7 +26,7 @@ MUTATIONS = [
      "rel = (a[None, :] - a[:, None] + M - 1) * (2 * M - 1) + (c[None, :] - c[:, None] + M - 1)"),
     ("rel-row-col-swapped", "rel = (a[:, None] - a[None, :] + M - 1) * (2 * M - 1) + (c[:, None] - c[None, :] + M - 1)",
      "rel = (c[:, None] - c[None, :] + M - 1) * (2 * M - 1) + (a[:, None] - a[None, :] + M - 1)"),
-    ("scale-dropped", "scale = float(d) ** -0.5", "scale = 1.0"),
+    ("scale-dropped", "scale = float(dq) ** -0.5", "scale = 1.0"),
     ("softmax-over-queries", "Smax = S.max(axis=-1, keepdims=True)\n        E = np.exp(S - Smax)\n        P = E / E.sum(axis=-1, keepdims=True)",
      "Smax = S.max(axis=-2, keepdims=True)\n        E = np.exp(S - Smax)\n        P = E / E.sum(axis=-2, keepdims=True)"),
     ("bias-head-offset", "S = S + table[rel][:, :, h0:h0 + gh].transpose(2, 0, 1)[None]", "S = S + table[rel][:, :, 0:gh].transpose(2, 0, 1)[None]"),
@@ -39,9 +39,9 @@ MUTATIONS = [
     ("bwd-dv-uses-dS", 'dvw = np.einsum("nhpq,nphd->nqhd", P, dO)', 'dvw = np.einsum("nhpq,nphd->nqhd", dS if False else P.transpose(0, 1, 3, 2), dO)'),
     ("bwd-dtable-head", "np.add.at(dtable[:, h0 + hh], rel.ravel(), dSh[hh].ravel())", "np.add.at(dtable[:, hh], rel.ravel(), dSh[hh].ravel())"),
     ("bwd-dtable-transposed", "np.add.at(dtable[:, h0 + hh], rel.ravel(), dSh[hh].ravel())", "np.add.at(dtable[:, h0 + hh], rel.T.ravel(), dSh[hh].ravel())"),
-    ("bwd-dwproj-transposed", "dw_proj = dy2.T @ A.reshape(-1, C)", "dw_proj = A.reshape(-1, C).T @ dy2"),
-    ("bwd-reverse-shift-dropped", "dst[..., ch] = reverse_shift(window_reverse(src.reshape(-1, N, gh * d), M, B, H, W), s)",
-     "dst[..., ch] = window_reverse(src.reshape(-1, N, gh * d), M, B, H, W)"),
+    ("bwd-dwproj-transposed", "dw_proj = dy2.T @ A.reshape(-1, A.shape[-1])", "dw_proj = A.reshape(-1, A.shape[-1]).T @ dy2"),
+    ("bwd-reverse-shift-dropped", "dst[..., sl] = reverse_shift(window_reverse(src.reshape(-1, N, gh * wd), M, B, H, W), s)",
+     "dst[..., sl] = window_reverse(src.reshape(-1, N, gh * wd), M, B, H, W)"),
     ("bwd-dx-weight-transposed", "dx = (dqkv @ w_qkv).reshape(B, H, W, C)", "dx = (dqkv @ w_qkv[:, ::-1]).reshape(B, H, W, C)"),
 ]
 

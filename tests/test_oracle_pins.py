@@ -284,3 +284,91 @@ def test_gradient_invariants():
     assert np.abs(g["db_qkv"][C:2 * C]).max() < 1e-12
     assert np.allclose(g["db_proj"], dy.reshape(-1, C).sum(0), atol=1e-12)
     assert np.abs(g["db_qkv"][:C]).max() > 1e-3 and np.abs(g["db_qkv"][2 * C:]).max() > 1e-3
+
+
+# ---------------------------------------------------------------- narrowed Q/K projections (Sec. "Parameter Allocation")
+def _narrow_params(rng, C, nh, M, dq, dv, wstd=0.3):
+    Cq, Cv = nh * dq, nh * dv
+    return (rng.standard_normal((2 * Cq + Cv, C)) * wstd, rng.standard_normal(2 * Cq + Cv) * 0.2,
+            rng.standard_normal((C, Cv)) * wstd, rng.standard_normal(C) * 0.2, rng.standard_normal(((2 * M - 1) ** 2, nh)) * 0.5)
+
+
+@pytest.mark.parametrize("dq,dv", [(1, 2), (3, 2), (2, 5)])
+def test_narrow_projections_against_bruteforce_global_attention(dq, dv):
+    rng = np.random.default_rng(31)
+    B, H, W, C, nh, M = 1, 8, 8, 8, 4, 4
+    x = rng.standard_normal((B, H, W, C))
+    prm = _narrow_params(rng, C, nh, M, dq, dv)
+    y, _ = orc.forward(x, *prm, M, (1, 3), (0, 1), qk_dim=dq, v_dim=dv)
+    yb = orc.bruteforce_forward(x, *prm, M, (1, 3), (0, 1), qk_dim=dq, v_dim=dv)
+    assert y.shape == x.shape
+    assert np.abs(y - yb).max() <= 1e-12 * max(1.0, np.abs(yb).max())
+
+
+def test_narrow_layer_equals_full_width_layer_with_zero_rows():
+    """A layer with qk_dim = k < d is the full-width layer whose Q,K rows beyond k are zero and whose Q rows are
+    rescaled by sqrt(d / k) (the full layer divides the scores by sqrt(d), the narrow one by sqrt(k)).  The
+    gradients of the shared rows agree likewise (those of the rescaled Q rows up to that factor)."""
+    rng = np.random.default_rng(37)
+    B, H, W, C, nh, M, k = 2, 8, 8, 12, 3, 4, 2
+    d = C // nh
+    x = rng.standard_normal((B, H, W, C))
+    dy = rng.standard_normal((B, H, W, C))
+    w, b, wp, bp, table = _narrow_params(rng, C, nh, M, k, d)
+    Cq = nh * k
+    full_w = np.zeros((3 * C, C))
+    full_b = np.zeros(3 * C)
+    f = np.sqrt(d / k)
+    rows_q, rows_k = [], []
+    for h in range(nh):
+        for c in range(k):
+            rows_q.append(h * d + c)
+            rows_k.append(C + h * d + c)
+    full_w[rows_q] = w[:Cq] * f
+    full_b[rows_q] = b[:Cq] * f
+    full_w[rows_k] = w[Cq:2 * Cq]
+    full_b[rows_k] = b[Cq:2 * Cq]
+    full_w[2 * C:] = w[2 * Cq:]
+    full_b[2 * C:] = b[2 * Cq:]
+    gh, gs = (1, 2), (0, 2)
+    y, cache = orc.forward(x, w, b, wp, bp, table, M, gh, gs, qk_dim=k)
+    g = orc.backward(cache, dy)
+    yf, cachef = orc.forward(x, full_w, full_b, wp, bp, table, M, gh, gs)
+    gf = orc.backward(cachef, dy)
+    assert np.abs(y - yf).max() <= 1e-13
+    assert np.abs(g["dx"] - gf["dx"]).max() <= 1e-12
+    assert np.abs(g["dw_qkv"][:Cq] - gf["dw_qkv"][rows_q] * f).max() <= 1e-11
+    assert np.abs(g["dw_qkv"][Cq:2 * Cq] - gf["dw_qkv"][rows_k]).max() <= 1e-11
+    assert np.abs(g["dw_qkv"][2 * Cq:] - gf["dw_qkv"][2 * C:]).max() <= 1e-11
+    assert np.abs(g["db_qkv"][:Cq] - gf["db_qkv"][rows_q] * f).max() <= 1e-11
+    assert np.abs(g["dbias_table"] - gf["dbias_table"]).max() <= 1e-11
+    assert np.abs(g["dw_proj"] - gf["dw_proj"]).max() <= 1e-11
+
+
+def test_narrow_projection_gradients_match_finite_differences():
+    rng = np.random.default_rng(41)
+    B, H, W, C, nh, M, dq, dv = 1, 8, 8, 6, 3, 4, 3, 4
+    x = rng.standard_normal((B, H, W, C))
+    dy = rng.standard_normal((B, H, W, C))
+    prm = list(_narrow_params(rng, C, nh, M, dq, dv))
+    gh, gs = (2, 1), (1, 0)
+    _, cache = orc.forward(x, *prm, M, gh, gs, qk_dim=dq, v_dim=dv)
+    g = orc.backward(cache, dy)
+    names = ["w_qkv", "b_qkv", "w_proj", "b_proj", "bias_table"]
+    grads = {"x": g["dx"], "w_qkv": g["dw_qkv"], "b_qkv": g["db_qkv"], "w_proj": g["dw_proj"], "b_proj": g["db_proj"],
+             "bias_table": g["dbias_table"]}
+    tensors = dict(zip(names, prm))
+    tensors["x"] = x
+    eps = 1e-6
+    for name, t in tensors.items():
+        for _ in range(2):
+            dirn = rng.standard_normal(t.shape)
+
+            def at(step):
+                xx = x + step * dirn if name == "x" else x
+                pp = [p + step * dirn if n == name else p for n, p in zip(names, prm)]
+                yy, _ = orc.forward(xx, *pp, M, gh, gs, keep=False, qk_dim=dq, v_dim=dv)
+                return float((yy * dy).sum())
+            fd = (at(eps) - at(-eps)) / (2 * eps)
+            an = float((grads[name] * dirn).sum())
+            assert abs(fd - an) <= 2e-7 * max(1.0, abs(an)), (name, fd, an)

@@ -2,9 +2,12 @@
 inside an application that owns all of it, a C program with no GPU allocator, a loop where cudaMalloc's
 device-wide synchronisation is not acceptable).  Its intermediates live in a fixed array inside the
 library's device image instead of a caller-provided scratch buffer.  Called through the C ABI twice in
-a row, it must give what gswa_forward gives in inference mode (same tolerance as the parity tests), the
-second call included, since every call reuses the array with the previous call's contents still in it.
+a row, it must give what the fp64 CPU checker gives (same tolerance as the parity tests) and, bit for bit,
+what gswa_forward gives in inference mode, the second call included, since every call reuses the array
+with the previous call's contents still in it; and it must leave the amount of free device memory alone.
 Collected last on purpose, so that a run which stops at the first failure has already run the rest."""
+import ctypes
+
 import numpy as np
 import pytest
 
@@ -12,7 +15,7 @@ from paper_2409_06206_b200 import binding as gb
 from paper_2409_06206_b200 import build as gbuild
 from paper_2409_06206_b200.inputs import LayerConfig, make_inputs
 
-from gpu_util import TOL, rel_err, run_gpu, to_device
+from gpu_util import TOL, rel_err, run_gpu, run_oracle, to_device
 
 pytestmark = pytest.mark.gpu
 
@@ -27,23 +30,37 @@ def _built():
     gbuild.build()
 
 
+def _free_device_bytes() -> int:
+    import torch
+    return torch.cuda.mem_get_info()[0]
+
+
 @pytest.mark.parametrize("cfg", CASES, ids=[c.name for c in CASES])
-def test_static_scratch_forward_matches_forward_twice(cfg):
+def test_static_scratch_forward_matches_checker_and_forward_twice(cfg):
     import torch
     inp = make_inputs(cfg)
     inp2 = make_inputs(LayerConfig(**{**cfg.__dict__, "seed": cfg.seed + 100}))
     desc = gb.Desc.from_config(cfg)
     tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
-    for which in (inp, inp2):                      # two calls in a row, different data each time
-        ref = run_gpu(cfg, which, backward=False, inference=True)["y"]
+    for call, which in enumerate((inp, inp2)):     # two calls in a row, different data each time
+        ref = run_oracle(cfg, which, backward=False)["y"]
+        same = run_gpu(cfg, which, backward=False, inference=True)["y"]
         dev = {k: to_device(v, cfg.dtype) for k, v in which.items()}
         y = torch.full(which["x"].shape, float("nan"), dtype=tdt, device="cuda")
+        torch.cuda.synchronize()
+        free0, alloc0, reserved0 = _free_device_bytes(), torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
         gb.gswa_forward_static(desc, dev["x"], dev["w_qkv"], dev["b_qkv"], dev["w_proj"], dev["b_proj"],
                                dev["bias_table"], y)
-        torch.cuda.synchronize()
+        gb.gswa_static_status()                    # waits for the stream; raises if a kernel gave up a wait
+        if call == 1:
+            # the property the entry point exists for: by the second call (the first may have made the driver load
+            # kernels) nothing is taken from, or returned to, the device's memory, by this library or through torch
+            assert _free_device_bytes() == free0
+            assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
         got = y.float().cpu().numpy().astype(np.float64)
         assert np.isfinite(got).all()
         assert rel_err(got, ref) <= TOL[cfg.dtype]
+        assert rel_err(got, same) == 0.0
 
 
 def test_static_scratch_rejects_layers_beyond_its_size():
