@@ -172,6 +172,7 @@ bool fast_path_ok(const Plan& p) {
   if (p.dqk != p.d || p.dv != p.d) return false;             // narrowed Q/K projections run on the shape-generic kernels
   if (p.M != 8 || p.d > 32 || (p.d & 1) || (p.C & 3) || p.C > 252 || p.G > 4) return false;
   if (p.nh * (p.d <= 16 ? 16 : 32) < 64) return false;       // padded rows must fill one TMA box of 64 columns
+  if (p.nh * (p.d <= 16 ? 16 : 32) > 256) return false;      // the padded attention width is the N extent of one MMA (dW_proj)
   if (p.T >= (1LL << 30) / 4) return false;
   Plan q = p;
   q.dp = p.d <= 16 ? 16 : 32;

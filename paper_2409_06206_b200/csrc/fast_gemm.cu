@@ -863,6 +863,7 @@ int launch_gt(const GTLaunch& L, int nsplits, cudaStream_t st, const char* name)
 
 int launch_gr(const GRLaunch& L, cudaStream_t st, const char* name) {
   GRLaunch Lc = L;
+  if (L.NP > 256 || L.NP % 64 != 0) return GSWA_ERR_UNSUPPORTED;      // N extent of one tcgen05.mma
   if (Lc.mbpc < 1 || Lc.mbpc * L.NP > 512) Lc.mbpc = 1;
   // 16-byte copies need 16-byte aligned sources: the base, and a row pitch of 0 (every row) or 8 (even rows) mod 16
   Lc.p16 = (reinterpret_cast<uintptr_t>(L.P) & 15) != 0 ? 0 : ((L.ldp * 2) % 16 == 0 ? 2 : ((L.ldp * 2) % 16 == 8 ? 1 : 0));
