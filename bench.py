@@ -251,7 +251,7 @@ def timed_repeats(args, step, barrier, check_status, gb):
         e1.record()
         barrier()
         launches = gb.gswa_launch_count() - n0
-        check_status()                                   # raises on GSWA_ERR_DEVICE
+        check_status()                                   # raises on GSWA_ERR_DEVICE (outside the timed region)
         per_step.append(max_over_ranks(e0.elapsed_time(e1)) / args.steps)
     t1 = time.perf_counter()
     return float(np.median(per_step)), per_step, int(launches), t0, t1
@@ -306,14 +306,23 @@ def run_ours(args, cfg):
                          dev["dy"], dx, grads["dw_qkv"], grads["db_qkv"], grads["dw_proj"], grads["db_proj"],
                          grads["dbias_table"], scratch)
 
+    def check_status():
+        # the backward call clears the error word its forward call may have set (they share `scratch`), so the
+        # forward pass is checked on its own first
+        gb.gswa_forward(desc, dev["x"], dev["w_qkv"], dev["b_qkv"], dev["w_proj"], dev["b_proj"], dev["bias_table"], y,
+                        saved, scratch)
+        gb.gswa_scratch_status(desc, scratch)
+        step()
+        gb.gswa_scratch_status(desc, scratch)
+
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
-    gb.gswa_scratch_status(desc, scratch)
+    check_status()
     fused_peak = torch.cuda.max_memory_allocated() - mem0
     sampler = ClockSampler(local) if rank == 0 else None
     time.sleep(0.25 if rank == 0 else 0.0)
-    ms_step, ms_repeats, launches, t0, t1 = timed_repeats(args, step, barrier, lambda: gb.gswa_scratch_status(desc, scratch), gb)
+    ms_step, ms_repeats, launches, t0, t1 = timed_repeats(args, step, barrier, check_status, gb)
     clocks = sampler.stop(t0, t1) if sampler else None
     value = world * cfg.tokens / (ms_step * 1e-3)
 

@@ -69,7 +69,8 @@ enum {
   /* (No flag asks for bitwise-reproducible reductions: the float32 parameter gradients are accumulated with
    *  atomics on every path, see gswa_backward.) */
   GSWA_FLAG_FUSED_FWD = 4u,  /* tensor-core path: one kernel for QKV projection + forward attention (slower at C = 180; kept as a measured alternative) */
-  GSWA_FLAG_TCGEN05_ATTN = 8u /* tensor-core path: attention backward on tcgen05 with TMEM accumulators instead of warp-level mma.sync (4 % slower at C = 180; kept as a measured alternative) */
+  GSWA_FLAG_TCGEN05_ATTN = 8u, /* tensor-core path: attention backward on tcgen05 with TMEM accumulators instead of warp-level mma.sync (4 % slower at C = 180; kept as a measured alternative) */
+  GSWA_FLAG_COPY_LOADERS = 16u /* tensor-core path: feed the window-order GEMMs with 8/16-byte asynchronous copies into a shared-memory operand (the path layers with odd shifts take anyway) instead of bulk copies + a TMEM A operand */
 };
 
 /* Layer description (host memory, read during the call only). */

@@ -15,7 +15,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libgswa.so")
 
 GSWA_F32, GSWA_BF16 = 0, 1
-FLAG_ACCUMULATE, FLAG_GENERIC, FLAG_FUSED_FWD, FLAG_TCGEN05_ATTN = 1, 2, 4, 8
+FLAG_ACCUMULATE, FLAG_GENERIC, FLAG_FUSED_FWD, FLAG_TCGEN05_ATTN, FLAG_COPY_LOADERS = 1, 2, 4, 8, 16
 
 STATIC_SCRATCH_BYTES = 16 << 20
 

@@ -51,6 +51,25 @@ int make_units(const Plan& p, Unit* units, int cap) {
   return n;
 }
 
+// Units of the window GEMM with its A operand in tensor memory: whole head groups where the weight image, the
+// accumulators and the row stages fit one SM, else the group cut into equal parts.  `nb` = output blocks per head.
+int make_units_tm(const Plan& p, Unit* units, int nb, int cap) {
+  int n = 0;
+  for (int g = 0; g < p.G; ++g) {
+    const int want = p.gh[g] < cap ? p.gh[g] : cap;
+    const int hpu = gwt_heads_per_unit(p.Cp, p.dp, p.C, nb, want);
+    if (hpu == 0) return -1;
+    const int parts = (p.gh[g] + hpu - 1) / hpu;
+    for (int i = 0, h = 0; i < parts; ++i) {
+      const int take = (p.gh[g] - h + (parts - i) - 1) / (parts - i);
+      if (n == kMaxUnits) return -1;
+      units[n++] = Unit{g, p.gh0[g] + h, take};
+      h += take;
+    }
+  }
+  return n;
+}
+
 // Split of the output columns of a token GEMM with K = kvalid so that the resident weight image,
 // the staging tile and at least three ring stages fit.
 bool token_split(int C, int K, TokenSplit* ts) {
@@ -267,10 +286,20 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
                  const void* b_proj, const void* table, void* y, void* saved, void* scratch, bool want_L,
                  cudaStream_t st) {
   using bf = __nv_bfloat16;
-  Unit units[kMaxUnits];
-  const int nu = make_units(p, units, 2);
+  // Units of the attention kernels when the layer has more heads than one-head units fit (cap 2), and of the QKV
+  // GEMM: whole groups with the A operand in tensor memory where the rows can be fetched by bulk copies, else
+  // units of at most two heads fed by the copy loaders.
+  Unit units2[kMaxUnits], units[kMaxUnits];
+  const int nu2 = make_units(p, units2, 2);
+  const bool tm = !(p.flags & (GSWA_FLAG_FUSED_FWD | GSWA_FLAG_COPY_LOADERS)) && gwt_usable(x, p.C, p.H, p.W, p.gs, p.G);
+  int nu = tm ? make_units_tm(p, units, 3, kMaxHeads) : -1;
+  const bool use_tm = nu > 0;
+  if (!use_tm) {
+    nu = nu2;
+    for (int i = 0; i < nu2; ++i) units[i] = units2[i];
+  }
   TokenSplit tp;
-  if (nu <= 0 || !token_split(p.C, p.Ap, &tp)) return GSWA_ERR_UNSUPPORTED;
+  if (nu <= 0 || nu2 <= 0 || !token_split(p.C, p.Ap, &tp)) return GSWA_ERR_UNSUPPORTED;
   const FwdScratch fs = fwd_layout(p, units, nu, tp);
   const FastGeom geo = make_geom(p);
   char* sc = static_cast<char*>(scratch);
@@ -354,16 +383,17 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
       w.ones_col = fold_bias ? 1 : 0;
       w.out = qkv + geo.qkv_off[u.g] + (long long)(u.h0 - p.gh0[u.g]) * 3 * 64 * p.dp;
       w.win_stride = (long long)p.gh[u.g] * 3 * 64 * p.dp;
-      // one accumulator chunk per unit when its columns fit one MMA (N <= 256), else one per head
-      if (u.nheads * 3 * p.dp <= 256) { w.nchunks = 1; w.cw = u.nheads * 3 * p.dp; }
+      // copy loaders: one accumulator chunk per unit when its columns fit one MMA (N <= 256), else one per head;
+      // A operand in tensor memory: one chunk per head (the chunks of a tile are drained while the next ones fill)
+      if (!use_tm && u.nheads * 3 * p.dp <= 256) { w.nchunks = 1; w.cw = u.nheads * 3 * p.dp; }
       else { w.nchunks = u.nheads; w.cw = 3 * p.dp; }
       w.q_every3 = 1;
       w.qscale = qscale;
     }
-    if ((rc = launch_gw(gw, nu, p.Cp, p.dp, st, "qkv_gemm"))) return rc;
+    if ((rc = use_tm ? launch_gwt(gw, nu, p.Cp, p.dp, st, "qkv_gemm") : launch_gw(gw, nu, p.Cp, p.dp, st, "qkv_gemm"))) return rc;
 
     AttnLaunch al{};
-    attn_units(p, geo, units, nu, &al);
+    attn_units(p, geo, units2, nu2, &al);
     al.qkv = qkv; al.table = (const bf*)table; al.A = A; al.Lt = want_L ? Lt : nullptr; al.err = err;
     al.scale = 1.0f / sqrtf((float)p.d);
     if ((rc = launch_attn_fwd(al, st))) return rc;
@@ -480,6 +510,9 @@ int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w
     w.win_stride = (long long)p.gh[u.g] * 64 * p.dp;
     w.nchunks = 1; w.cw = u.nheads * p.dp; w.q_every3 = 0; w.qscale = 1.f;
   }
+  // (dO = dy W^P has few columns per tile: with the A operand in tensor memory its tile period is set by the load
+  // latency of the two tiles it keeps in flight, 87 us against 62 us for the copy-fed kernel at C = 180, so the
+  // backward pass keeps the copy loaders)
   if ((rc = launch_gw(gw, nu, p.Cp, p.dp, st, "dattn_gemm"))) return finish(rc);
 
   al.qkv = qkv; al.table = (const bf*)table; al.Lt = const_cast<float*>(Lt); al.dO = dO; al.dqkv = dqkv;

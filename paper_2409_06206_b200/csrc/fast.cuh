@@ -65,7 +65,7 @@ struct GWUnit {
 struct GWLaunch {
   GWUnit u[kMaxUnits];
   int* err;
-  int nslots;                  // ring slots of 16 KB (set by launch_gw)
+  int nslots;                  // ring slots of 16 KB (set by launch_gw) / quarter-tile stages (set by launch_gwt)
   int cta0[kMaxUnits + 1];     // first CTA of every unit (set by launch_gw)
 };
 
@@ -112,6 +112,11 @@ struct GRLaunch {
 };
 
 int launch_gw(const GWLaunch& L, int nunits, int Cp, int dp, cudaStream_t st, const char* name);
+// The same GEMM with the A operand in tensor memory (fast_gemm_tm.cu): rows arrive by bulk copies of whole window
+// rows, which needs every piece of a window row to start and end on a 16-byte boundary (gwt_usable).
+bool gwt_usable(const void* A, int lda, int H, int W, const int* shifts, int nshifts);
+int gwt_heads_per_unit(int Cp, int dp, int C, int nb, int cap);   // nb = output blocks of dp columns per head (3: q,k,v; 1: dO)
+int launch_gwt(const GWLaunch& L, int nunits, int Cp, int dp, cudaStream_t st, const char* name);
 
 // ---- fused forward: QKV projection of a window pair on the tensor core, its q,k,v tiles handed to the
 // attention warps of the same CTA through shared memory (and, for training, shipped to `qkv_out`).

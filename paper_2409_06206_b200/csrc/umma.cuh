@@ -75,6 +75,16 @@ __device__ __forceinline__ void mma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, ui
       : "memory");
 }
 
+// One lane of a converged warp, chosen by the hardware.  A warp that runs its MMA loop with all lanes (uniform
+// control flow, uniform descriptor arithmetic) and predicates only the tcgen05 instructions with this keeps the
+// operands in uniform registers; a loop under `if (lane == 0)` is divergent code and pays a register-to-uniform move
+// per operand per instruction.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}\n" : "=r"(pred));
+  return pred != 0;
+}
+
 // Makes the mbarrier track completion of all tcgen05.mma issued so far by this thread.
 __device__ __forceinline__ void commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
@@ -137,6 +147,10 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
       "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]),
       "r"(v[31])
       : "memory");
+}
+// 8 bytes from shared memory (32-bit shared-space address).
+__device__ __forceinline__ void lds64(uint32_t& a, uint32_t& b, uint32_t addr) {
+  asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(a), "=r"(b) : "r"(addr) : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 

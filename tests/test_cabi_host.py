@@ -82,6 +82,7 @@ def test_binding_constants_match_the_header():
     assert int(vals["GSWA_FLAG_GENERIC"]) == gb.FLAG_GENERIC
     assert int(vals["GSWA_FLAG_FUSED_FWD"]) == gb.FLAG_FUSED_FWD
     assert int(vals["GSWA_FLAG_TCGEN05_ATTN"]) == gb.FLAG_TCGEN05_ATTN
+    assert int(vals["GSWA_FLAG_COPY_LOADERS"]) == gb.FLAG_COPY_LOADERS
     assert int(vals["GSWA_F32"]) == gb.GSWA_F32 and int(vals["GSWA_BF16"]) == gb.GSWA_BF16
     m = re.search(r"GSWA_STATIC_SCRATCH_BYTES \((\d+)u << (\d+)\)", text)
     assert int(m.group(1)) << int(m.group(2)) == gb.STATIC_SCRATCH_BYTES

@@ -184,10 +184,11 @@ def test_random_shapes_tensor_core_path(cfg):
     assert_close(run_gpu(cfg, inp), ref, cfg.dtype)
     assert_close(run_gpu(cfg, inp, flags=gb.FLAG_FUSED_FWD), ref, cfg.dtype)
     assert_close(run_gpu(cfg, inp, flags=gb.FLAG_TCGEN05_ATTN), ref, cfg.dtype)
+    assert_close(run_gpu(cfg, inp, flags=gb.FLAG_COPY_LOADERS), ref, cfg.dtype)
 
 
-@pytest.mark.parametrize("flags", [0, gb.FLAG_FUSED_FWD, gb.FLAG_TCGEN05_ATTN, gb.FLAG_GENERIC],
-                         ids=["default", "fused-fwd", "tcgen05-attn", "generic"])
+@pytest.mark.parametrize("flags", [0, gb.FLAG_FUSED_FWD, gb.FLAG_TCGEN05_ATTN, gb.FLAG_COPY_LOADERS, gb.FLAG_GENERIC],
+                         ids=["default", "fused-fwd", "tcgen05-attn", "copy-loaders", "generic"])
 @pytest.mark.parametrize("cfg", EXCITED, ids=[c.name for c in EXCITED])
 def test_score_exciting_inputs(cfg, flags):
     """Weights ~ N(0, 1/C) and a table of std 0.7: the softmax is far from uniform, so the bias gather, the query
