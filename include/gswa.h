@@ -178,6 +178,34 @@ int gswa_debug_index_maps(const gswa_desc* desc, int32_t group, int32_t* win_id,
  * GSWA_ERR_UNSUPPORTED for layers off the tensor-core path (they keep no error word). */
 int gswa_debug_expire_wait(const gswa_desc* desc, void* scratch, void* cuda_stream);
 
+/* ---- The layer around GSWA (Sec. "Agile Swin Transformer Block", Eq. 4 and Eq. 5):
+ *        X1 = GSWA(LN(X)) + X,    X2 = MLP(LN(X1)) + X1.
+ * LayerNorm is taken over the C channels of each token (biased variance, eps = 1e-5, learnable scale and shift);
+ * the MLP is FC1 [mlp_hidden, C] -> GELU (exact Gaussian-CDF form) -> FC2 [C, mlp_hidden].  mlp_hidden == 0 stops
+ * after Eq. 4 (the output is X1 and the second LayerNorm / MLP pointers are ignored).  All pointers of both
+ * structures are DEVICE pointers; parameters have the element type `dtype`, gradients are float32 and every one of
+ * them is required (overwritten unless GSWA_FLAG_ACCUMULATE).  `saved` / `scratch` follow gswa_forward /
+ * gswa_backward: sizes from gswa_astl_workspace_query, `saved` NULL = inference (scratch of infer_scratch_bytes).
+ * The device error word of the tensor-core attention kernels is at the head of `scratch` (gswa_scratch_status). */
+typedef struct gswa_astl_params {
+  const void *ln1_g, *ln1_b;                                    /* [C]                                   */
+  const void *w_qkv, *b_qkv, *w_proj, *b_proj, *bias_table;     /* as for gswa_forward (b_* may be NULL) */
+  const void *ln2_g, *ln2_b;                                    /* [C]                                   */
+  const void *w_fc1, *b_fc1;                                    /* [mlp_hidden, C], [mlp_hidden]         */
+  const void *w_fc2, *b_fc2;                                    /* [C, mlp_hidden], [C]                  */
+} gswa_astl_params;
+typedef struct gswa_astl_grads {
+  float *dln1_g, *dln1_b, *dw_qkv, *db_qkv, *dw_proj, *db_proj, *dbias_table;
+  float *dln2_g, *dln2_b, *dw_fc1, *db_fc1, *dw_fc2, *db_fc2;
+} gswa_astl_grads;
+int gswa_astl_workspace_query(const gswa_desc* desc, int32_t mlp_hidden, size_t* saved_bytes, size_t* fwd_scratch_bytes,
+                              size_t* infer_scratch_bytes, size_t* bwd_scratch_bytes);
+int gswa_astl_forward(const gswa_desc* desc, int32_t mlp_hidden, const void* x, const gswa_astl_params* params, void* y,
+                      void* saved, void* scratch, size_t scratch_bytes, void* cuda_stream);
+int gswa_astl_backward(const gswa_desc* desc, int32_t mlp_hidden, const void* x, const gswa_astl_params* params,
+                       const void* saved, const void* dy, void* dx, const gswa_astl_grads* grads, void* scratch,
+                       size_t scratch_bytes, void* cuda_stream);
+
 /* One training step on HOST buffers: copies x, the parameters and dy to the device arena, runs
  * gswa_forward + gswa_backward, copies y, dx and the parameter gradients back, and waits for the
  * stream.  All tensor pointers are HOST pointers (pinned memory makes the copies asynchronous);

@@ -20,6 +20,7 @@ FLAG_ACCUMULATE, FLAG_GENERIC, FLAG_FUSED_FWD, FLAG_TCGEN05_ATTN, FLAG_COPY_LOAD
 STATIC_SCRATCH_BYTES = 16 << 20
 
 EXPORTS = ("gswa_workspace_query", "gswa_forward", "gswa_forward_static", "gswa_static_status", "gswa_backward",
+           "gswa_astl_workspace_query", "gswa_astl_forward", "gswa_astl_backward",
            "gswa_index_maps", "gswa_debug_index_maps", "gswa_debug_expire_wait", "gswa_step_host", "gswa_scratch_status", "gswa_profile_enable", "gswa_profile_read", "gswa_launch_count", "gswa_status_string")
 
 
@@ -34,6 +35,20 @@ class _Desc(C.Structure):
                 ("window", C.c_int32), ("num_groups", C.c_int32), ("group_heads", C.POINTER(C.c_int32)),
                 ("group_shift", C.POINTER(C.c_int32)), ("dtype", C.c_int32), ("qk_dim", C.c_int32),
                 ("v_dim", C.c_int32), ("flags", C.c_uint32)]
+
+
+ASTL_PARAMS = ("ln1_g", "ln1_b", "w_qkv", "b_qkv", "w_proj", "b_proj", "bias_table", "ln2_g", "ln2_b", "w_fc1", "b_fc1",
+               "w_fc2", "b_fc2")
+ASTL_GRADS = ("dln1_g", "dln1_b", "dw_qkv", "db_qkv", "dw_proj", "db_proj", "dbias_table", "dln2_g", "dln2_b", "dw_fc1",
+              "db_fc1", "dw_fc2", "db_fc2")
+
+
+class _AstlParams(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ASTL_PARAMS]
+
+
+class _AstlGrads(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ASTL_GRADS]
 
 
 class Desc:
@@ -90,6 +105,11 @@ def lib() -> C.CDLL:
         L.gswa_scratch_status.restype = C.c_int
         L.gswa_static_status.argtypes = [vp]
         L.gswa_static_status.restype = C.c_int
+        L.gswa_astl_workspace_query.argtypes = [dp, C.c_int32, szp, szp, szp, szp]
+        L.gswa_astl_forward.argtypes = [dp, C.c_int32, vp, C.POINTER(_AstlParams), vp, vp, vp, sz, vp]
+        L.gswa_astl_backward.argtypes = [dp, C.c_int32, vp, C.POINTER(_AstlParams), vp, vp, vp, C.POINTER(_AstlGrads), vp, sz, vp]
+        for name in ("gswa_astl_workspace_query", "gswa_astl_forward", "gswa_astl_backward"):
+            getattr(L, name).restype = C.c_int
         L.gswa_debug_index_maps.argtypes = [dp, C.c_int32] + [vp] * 5
         L.gswa_debug_index_maps.restype = C.c_int
         L.gswa_debug_expire_wait.argtypes = [dp, vp, vp]
@@ -170,6 +190,31 @@ def gswa_backward(desc: Desc, x, w_qkv, b_qkv, w_proj, bias_table, saved, dy, dx
 def gswa_index_maps(desc: Desc, group: int, win, slot, region, token_of, rel_index, stream=None) -> None:
     _check(lib().gswa_index_maps(C.byref(desc.c), group, _ptr(win), _ptr(slot), _ptr(region), _ptr(token_of),
                                  _ptr(rel_index), _stream(stream)))
+
+
+def gswa_astl_workspace_query(desc: Desc, mlp_hidden: int):
+    """-> (saved_bytes, fwd_scratch_bytes, infer_scratch_bytes, bwd_scratch_bytes) of the whole layer"""
+    out = [C.c_size_t(0) for _ in range(4)]
+    _check(lib().gswa_astl_workspace_query(C.byref(desc.c), mlp_hidden, *[C.byref(o) for o in out]))
+    return tuple(int(o.value) for o in out)
+
+
+def _astl_struct(cls, names, tensors):
+    return cls(*[_ptr(tensors.get(n)) for n in names])
+
+
+def gswa_astl_forward(desc: Desc, mlp_hidden: int, x, params: dict, y, saved, scratch, stream=None) -> None:
+    """params: name -> tensor for the names of ASTL_PARAMS (missing / None entries are passed as NULL)."""
+    q = _astl_struct(_AstlParams, ASTL_PARAMS, params)
+    _check(lib().gswa_astl_forward(C.byref(desc.c), mlp_hidden, _ptr(x), C.byref(q), _ptr(y), _ptr(saved), _ptr(scratch),
+                                   scratch.numel() * scratch.element_size(), _stream(stream)))
+
+
+def gswa_astl_backward(desc: Desc, mlp_hidden: int, x, params: dict, saved, dy, dx, grads: dict, scratch, stream=None) -> None:
+    q = _astl_struct(_AstlParams, ASTL_PARAMS, params)
+    g = _astl_struct(_AstlGrads, ASTL_GRADS, grads)
+    _check(lib().gswa_astl_backward(C.byref(desc.c), mlp_hidden, _ptr(x), C.byref(q), _ptr(saved), _ptr(dy), _ptr(dx),
+                                    C.byref(g), _ptr(scratch), scratch.numel() * scratch.element_size(), _stream(stream)))
 
 
 def gswa_debug_index_maps(desc: Desc, group: int, win_id, slot, region, rel_index, stream=None) -> None:

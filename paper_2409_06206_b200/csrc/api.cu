@@ -124,6 +124,57 @@ int make_plan(const gswa_desc* desc, Plan* p) {
 
 static bool misaligned(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) != 0; }
 
+// Argument checks and dispatch of one GSWA forward / backward for an already validated plan (shared by the plain
+// entry points and by the layer entry points of astl.cu, which add a skip connection through `resid`).
+int forward_impl(const Plan& p, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj, const void* b_proj,
+                 const void* bias_table, void* y, void* saved, void* scratch, size_t scratch_bytes, cudaStream_t st,
+                 const void* resid) {
+  if (!x || !w_qkv || !w_proj || !bias_table || !y) return GSWA_ERR_NULL;
+  if (p.T == 0) return GSWA_OK;
+  const size_t need = saved ? p.fwd_scratch : p.infer_scratch;
+  if (need > 0 && scratch == nullptr) return GSWA_ERR_NULL;
+  if (misaligned(x) || misaligned(w_qkv) || misaligned(b_qkv) || misaligned(w_proj) || misaligned(b_proj) ||
+      misaligned(bias_table) || misaligned(y) || misaligned(saved) || misaligned(scratch) || misaligned(resid))
+    return GSWA_ERR_ALIGN;
+  if (scratch_bytes < need) return GSWA_ERR_WORKSPACE;
+  if (p.fast) {
+    void* carry = saved ? saved : static_cast<char*>(scratch) + p.fwd_scratch;
+    return fast_forward(p, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, y, carry, scratch, saved != nullptr, st, resid);
+  }
+  void* carry = saved ? saved : scratch;
+  return generic_forward(p, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, y, carry, st, resid);
+}
+
+int backward_impl(const Plan& p, const void* x, const void* w_qkv, const void* w_proj, const void* bias_table,
+                  const void* saved, const void* dy, void* dx, float* dw_qkv, float* db_qkv, float* dw_proj, float* db_proj,
+                  float* dbias_table, void* scratch, size_t scratch_bytes, cudaStream_t st) {
+  if (!x || !w_qkv || !w_proj || !bias_table || !saved || !dy) return GSWA_ERR_NULL;
+  if (p.bwd_scratch > 0 && scratch == nullptr) return GSWA_ERR_NULL;
+  if (misaligned(x) || misaligned(w_qkv) || misaligned(w_proj) || misaligned(bias_table) || misaligned(saved) ||
+      misaligned(dy) || misaligned(dx) || misaligned(dw_qkv) || misaligned(db_qkv) || misaligned(dw_proj) ||
+      misaligned(db_proj) || misaligned(dbias_table) || misaligned(scratch))
+    return GSWA_ERR_ALIGN;
+  if (scratch_bytes < p.bwd_scratch) return GSWA_ERR_WORKSPACE;
+  int rc;
+  {
+    // one launch zeroes the parameter gradients (unless they accumulate) and, on the tensor-core path, the error
+    // word at the head of the scratch buffer
+    const size_t C = (size_t)p.C, Q = (size_t)p.Cqkv, Cv = (size_t)p.Cv, nrel = (size_t)(2 * p.M - 1) * (2 * p.M - 1);
+    const bool z = !(p.flags & GSWA_FLAG_ACCUMULATE);
+    float* const ptrs[6] = {z ? dw_qkv : nullptr, z ? db_qkv : nullptr, z ? dw_proj : nullptr, z ? db_proj : nullptr,
+                            z ? dbias_table : nullptr, p.fast && p.T > 0 ? static_cast<float*>(scratch) : nullptr};
+    const long long counts[6] = {(long long)(Q * C), (long long)Q, (long long)(C * Cv), (long long)C,
+                                 (long long)(nrel * p.nh), 64};
+    if ((rc = launch_zero(ptrs, counts, 6, st))) return rc;
+  }
+  if (p.T == 0) return GSWA_OK;
+  if (p.fast)
+    return fast_backward(p, x, w_qkv, w_proj, bias_table, saved, dy, dx, dw_qkv, db_qkv, dw_proj, db_proj, dbias_table,
+                         scratch, st);
+  return generic_backward(p, x, w_qkv, w_proj, bias_table, saved, dy, dx, dw_qkv, db_qkv, dw_proj, db_proj,
+                          dbias_table, scratch, st);
+}
+
 // Scratch of gswa_forward_static: part of the device image, so no allocation call is ever made for
 // it.  In host code this name is only a handle; the device address is looked up per device below.
 static __device__ __align__(256) unsigned char g_static_scratch[GSWA_STATIC_SCRATCH_BYTES];
@@ -173,24 +224,10 @@ int gswa_forward(const gswa_desc* desc, const void* x, const void* w_qkv, const 
                  const void* b_proj, const void* bias_table, void* y, void* saved, void* scratch,
                  size_t scratch_bytes, void* cuda_stream) {
   Plan p;
-  int rc = make_plan(desc, &p);
+  const int rc = make_plan(desc, &p);
   if (rc) return rc;
-  if (!x || !w_qkv || !w_proj || !bias_table || !y) return GSWA_ERR_NULL;
-  if (p.T == 0) return GSWA_OK;
-  const size_t need = saved ? p.fwd_scratch : p.infer_scratch;
-  if (need > 0 && scratch == nullptr) return GSWA_ERR_NULL;
-  if (misaligned(x) || misaligned(w_qkv) || misaligned(b_qkv) || misaligned(w_proj) || misaligned(b_proj) ||
-      misaligned(bias_table) || misaligned(y) || misaligned(saved) || misaligned(scratch))
-    return GSWA_ERR_ALIGN;
-  if (scratch_bytes < need) return GSWA_ERR_WORKSPACE;
-  if (p.T == 0) return GSWA_OK;
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  if (p.fast) {
-    void* carry = saved ? saved : static_cast<char*>(scratch) + p.fwd_scratch;
-    return fast_forward(p, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, y, carry, scratch, saved != nullptr, st);
-  }
-  void* carry = saved ? saved : scratch;
-  return generic_forward(p, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, y, carry, st);
+  return forward_impl(p, x, w_qkv, b_qkv, w_proj, b_proj, bias_table, y, saved, scratch, scratch_bytes,
+                      reinterpret_cast<cudaStream_t>(cuda_stream), nullptr);
 }
 
 int gswa_forward_static(const gswa_desc* desc, const void* x, const void* w_qkv, const void* b_qkv,
@@ -220,33 +257,10 @@ int gswa_backward(const gswa_desc* desc, const void* x, const void* w_qkv, const
                   size_t scratch_bytes, void* cuda_stream) {
   (void)b_qkv;
   Plan p;
-  int rc = make_plan(desc, &p);
+  const int rc = make_plan(desc, &p);
   if (rc) return rc;
-  if (!x || !w_qkv || !w_proj || !bias_table || !saved || !dy) return GSWA_ERR_NULL;
-  if (p.bwd_scratch > 0 && scratch == nullptr) return GSWA_ERR_NULL;
-  if (misaligned(x) || misaligned(w_qkv) || misaligned(w_proj) || misaligned(bias_table) || misaligned(saved) ||
-      misaligned(dy) || misaligned(dx) || misaligned(dw_qkv) || misaligned(db_qkv) || misaligned(dw_proj) ||
-      misaligned(db_proj) || misaligned(dbias_table) || misaligned(scratch))
-    return GSWA_ERR_ALIGN;
-  if (scratch_bytes < p.bwd_scratch) return GSWA_ERR_WORKSPACE;
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  {
-    // one launch zeroes the parameter gradients (unless they accumulate) and, on the tensor-core path, the error
-    // word at the head of the scratch buffer
-    const size_t C = (size_t)p.C, Q = (size_t)p.Cqkv, Cv = (size_t)p.Cv, nrel = (size_t)(2 * p.M - 1) * (2 * p.M - 1);
-    const bool z = !(p.flags & GSWA_FLAG_ACCUMULATE);
-    float* const ptrs[6] = {z ? dw_qkv : nullptr, z ? db_qkv : nullptr, z ? dw_proj : nullptr, z ? db_proj : nullptr,
-                            z ? dbias_table : nullptr, p.fast && p.T > 0 ? static_cast<float*>(scratch) : nullptr};
-    const long long counts[6] = {(long long)(Q * C), (long long)Q, (long long)(C * Cv), (long long)C,
-                                 (long long)(nrel * p.nh), 64};
-    if ((rc = launch_zero(ptrs, counts, 6, st))) return rc;
-  }
-  if (p.T == 0) return GSWA_OK;
-  if (p.fast)
-    return fast_backward(p, x, w_qkv, w_proj, bias_table, saved, dy, dx, dw_qkv, db_qkv, dw_proj, db_proj, dbias_table,
-                         scratch, st);
-  return generic_backward(p, x, w_qkv, w_proj, bias_table, saved, dy, dx, dw_qkv, db_qkv, dw_proj, db_proj,
-                          dbias_table, scratch, st);
+  return backward_impl(p, x, w_qkv, w_proj, bias_table, saved, dy, dx, dw_qkv, db_qkv, dw_proj, db_proj, dbias_table,
+                       scratch, scratch_bytes, reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
 int gswa_index_maps(const gswa_desc* desc, int32_t group, int32_t* win, int32_t* slot, int32_t* region,

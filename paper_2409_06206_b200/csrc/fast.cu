@@ -284,7 +284,7 @@ static void attn_units(const Plan& p, const FastGeom& geo, const Unit* units, in
 
 int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
                  const void* b_proj, const void* table, void* y, void* saved, void* scratch, bool want_L,
-                 cudaStream_t st) {
+                 cudaStream_t st, const void* resid) {
   using bf = __nv_bfloat16;
   // Units of the attention kernels when the layer has more heads than one-head units fit (cap 2), and of the QKV
   // GEMM: whole groups with the A operand in tensor memory where the rows can be fetched by bulk copies, else
@@ -402,7 +402,7 @@ int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_
   GTLaunch gt{};
   if ((rc = make_tmap(&gt.tmA, A, p.T, p.Ap, 128))) return rc;
   gt.natoms = tp.natoms; gt.rows = p.T;
-  gt.out = (bf*)y; gt.ldo = p.C; gt.NB = tp.NB; gt.nstages = tp.nstages; gt.stream_b = tp.stream_b; gt.err = err;
+  gt.out = (bf*)y; gt.ldo = p.C; gt.resid = (const bf*)resid; gt.NB = tp.NB; gt.nstages = tp.nstages; gt.stream_b = tp.stream_b; gt.err = err;
   for (int i = 0; i < tp.nsplit; ++i) {
     const int col0 = i * tp.NB;
     gt.s[i] = GTSplit{(const unsigned char*)sc + fs.pimg[i], fold_pbias || b_proj == nullptr ? nullptr : (const float*)(sc + fs.pbias[i]), col0,

@@ -81,6 +81,7 @@ struct GTLaunch {
   long long rows;
   __nv_bfloat16* out;
   int ldo;
+  const __nv_bfloat16* resid;  // or nullptr: packed rows [rows, ldo] added to the result (skip connection)
   int NB;                      // accumulator columns per CTA (multiple of 32, <= 256)
   int nstages;
   int stream_b;                // 1: the weight image travels through the ring with the A atoms (see gt_kernel)
@@ -211,7 +212,7 @@ bool fast_path_ok(const Plan& p);
 void fast_plan_sizes(Plan* p);
 int fast_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
                  const void* b_proj, const void* table, void* y, void* saved, void* scratch, bool want_L,
-                 cudaStream_t st);
+                 cudaStream_t st, const void* resid = nullptr);   // resid [B,H,W,C] or nullptr: added to y
 int fast_backward(const Plan& p, const void* x, const void* w_qkv, const void* w_proj, const void* table,
                   const void* saved, const void* dy, void* dx, float* dw_qkv, float* db_qkv, float* dw_proj,
                   float* db_proj, float* dtable, void* scratch, cudaStream_t st);

@@ -301,6 +301,13 @@ __global__ void __launch_bounds__(kThreads2, 1) gw_kernel(const __grid_constant_
 // gt_kernel
 // ==========================================================================================
 
+// Four bf16 sums in float arithmetic.
+__device__ __forceinline__ uint2 add_bf16x4(uint2 a, uint2 b) {
+  const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.x)), a1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.y));
+  const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.x)), b1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.y));
+  return make_uint2(pack_bf16(a0.x + b0.x, a0.y + b0.y), pack_bf16(a1.x + b1.x, a1.y + b1.y));
+}
+
 __global__ void __launch_bounds__(kThreads2, 1) gt_kernel(const __grid_constant__ GTLaunch L) {
   const GTSplit& sp = L.s[blockIdx.y];
   extern __shared__ unsigned char smem_raw[];
@@ -431,12 +438,26 @@ __global__ void __launch_bounds__(kThreads2, 1) gt_kernel(const __grid_constant_
       const unsigned char* sbase = mystg + lane * 8;
       const bool p0 = lane < n8, p1 = lane + 32 < n8;
       const int rend = nrows < 16 * half + 16 ? nrows : 16 * half + 16;
+      if (L.resid == nullptr) {
 #pragma unroll 4
-      for (int rr = 16 * half; rr < rend; ++rr) {
-        if (p0) *reinterpret_cast<uint2*>(obase + rr * obytes) = *reinterpret_cast<const uint2*>(sbase + rr * ncols * 2);
-        if (p1)
-          *reinterpret_cast<uint2*>(obase + rr * obytes + 256) =
-              *reinterpret_cast<const uint2*>(sbase + rr * ncols * 2 + 256);
+        for (int rr = 16 * half; rr < rend; ++rr) {
+          if (p0) *reinterpret_cast<uint2*>(obase + rr * obytes) = *reinterpret_cast<const uint2*>(sbase + rr * ncols * 2);
+          if (p1)
+            *reinterpret_cast<uint2*>(obase + rr * obytes + 256) =
+                *reinterpret_cast<const uint2*>(sbase + rr * ncols * 2 + 256);
+        }
+      } else {
+        // skip connection: the residual rows have the layout of the output rows
+        const char* const rbase = reinterpret_cast<const char*>(L.resid + trow0 * L.ldo + sp.col0) + lane * 8;
+#pragma unroll 4
+        for (int rr = 16 * half; rr < rend; ++rr) {
+          if (p0)
+            *reinterpret_cast<uint2*>(obase + rr * obytes) =
+                add_bf16x4(*reinterpret_cast<const uint2*>(sbase + rr * ncols * 2), __ldg(reinterpret_cast<const uint2*>(rbase + rr * obytes)));
+          if (p1)
+            *reinterpret_cast<uint2*>(obase + rr * obytes + 256) =
+                add_bf16x4(*reinterpret_cast<const uint2*>(sbase + rr * ncols * 2 + 256), __ldg(reinterpret_cast<const uint2*>(rbase + rr * obytes + 256)));
+        }
       }
     }
   }

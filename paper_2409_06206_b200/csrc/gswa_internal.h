@@ -40,6 +40,14 @@ struct HeadShifts {
 };
 
 int make_plan(const gswa_desc* desc, Plan* plan);
+// One GSWA forward / backward for a validated plan: pointer checks, then the tensor-core or the shape-generic path.
+// `resid` ([B,H,W,C] or nullptr) is added to y in the output projection's epilogue (skip connection of Eq. 4).
+int forward_impl(const Plan& p, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj, const void* b_proj,
+                 const void* bias_table, void* y, void* saved, void* scratch, size_t scratch_bytes, cudaStream_t st,
+                 const void* resid);
+int backward_impl(const Plan& p, const void* x, const void* w_qkv, const void* w_proj, const void* bias_table,
+                  const void* saved, const void* dy, void* dx, float* dw_qkv, float* db_qkv, float* dw_proj, float* db_proj,
+                  float* dbias_table, void* scratch, size_t scratch_bytes, cudaStream_t st);
 int check_launch();  // GSWA_OK or GSWA_ERR_CUDA (records the CUDA error text)
 int launch_zero(float* const* ptrs, const long long* counts, int nbuf, cudaStream_t st);   // one launch zeroes them all
 int device_sm_count();     // multiprocessors of the current device (148 if the query fails)
@@ -56,7 +64,8 @@ struct KernelScope {
 
 // ---- generic CUDA-core path (any shape the descriptor allows, f32 or bf16 storage, f32 arithmetic)
 int generic_forward(const Plan& p, const void* x, const void* w_qkv, const void* b_qkv, const void* w_proj,
-                    const void* b_proj, const void* table, void* y, void* saved, cudaStream_t st);
+                    const void* b_proj, const void* table, void* y, void* saved, cudaStream_t st,
+                    const void* resid = nullptr);   // resid [B,H,W,C] or nullptr: added to y (skip connection)
 int generic_backward(const Plan& p, const void* x, const void* w_qkv, const void* w_proj, const void* table,
                      const void* saved, const void* dy, void* dx, float* dw_qkv, float* db_qkv, float* dw_proj,
                      float* db_proj, float* dtable, void* scratch, cudaStream_t st);

@@ -97,7 +97,9 @@ def from_bf16_bits(b: np.ndarray) -> np.ndarray:
     return (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
 
 
-_TENSOR_STREAM = {"x": 1, "w_qkv": 2, "b_qkv": 3, "w_proj": 4, "b_proj": 5, "bias_table": 6, "dy": 7}
+_TENSOR_STREAM = {"x": 1, "w_qkv": 2, "b_qkv": 3, "w_proj": 4, "b_proj": 5, "bias_table": 6, "dy": 7,
+                  "ln1_g": 8, "ln1_b": 9, "ln2_g": 10, "ln2_b": 11, "w_fc1": 12, "b_fc1": 13, "w_fc2": 14, "b_fc2": 15,
+                  "w_heads": 16, "b_heads": 17}
 
 
 def _normal(seed: int, layer: int, name: str, shape, std: float) -> np.ndarray:
@@ -138,6 +140,41 @@ def make_inputs(cfg: LayerConfig, layer: int = 0, batch: int | None = None,
         if cfg.dtype == "bf16":
             a = round_to_bf16(a)
         out[name] = a
+    return out
+
+
+def make_layer_inputs(cfg: LayerConfig, mlp_hidden: int, layer: int = 0, batch: int | None = None) -> Dict[str, np.ndarray]:
+    """The tensors of one whole layer call (attention inside LayerNorm + skip, optionally followed by the MLP):
+    those of make_inputs plus LayerNorm scales ~ 1 + N(0, 0.1^2), shifts ~ N(0, 0.1^2), and the two
+    fully-connected layers ~ N(0, w_std^2) with biases ~ N(0, bias_std^2).  Here x is NOT normalised input: it is
+    drawn ~ N(0.5, 2^2) so that the LayerNorm has something to do."""
+    out = make_inputs(cfg, layer=layer, batch=batch)
+    C = cfg.C
+    out["x"] = (out["x"] * np.float32(2.0) + np.float32(0.5)).astype(np.float32)
+    shapes = {"ln1_g": ((C,), 0.1, 1.0), "ln1_b": ((C,), 0.1, 0.0), "ln2_g": ((C,), 0.1, 1.0), "ln2_b": ((C,), 0.1, 0.0),
+              "w_fc1": ((mlp_hidden, C), cfg.w_std, 0.0), "b_fc1": ((mlp_hidden,), cfg.bias_std, 0.0),
+              "w_fc2": ((C, mlp_hidden), cfg.w_std, 0.0), "b_fc2": ((C,), cfg.bias_std, 0.0)}
+    for name, (shape, std, mean) in shapes.items():
+        if 0 in shape:
+            continue
+        a = _normal(cfg.seed, layer, name, shape, std) if std > 0 else np.zeros(shape, np.float32)
+        out[name] = (a + np.float32(mean)).astype(np.float32)
+    if cfg.dtype == "bf16":
+        out = {k: round_to_bf16(v) for k, v in out.items()}
+    return out
+
+
+def make_sliced_inputs(cfg: LayerConfig, layer: int = 0, batch: int | None = None) -> Dict[str, np.ndarray]:
+    """The tensors of a channel-sliced layer call: per-head projections w_heads [heads, 2*qk + ds, ds] (ds = C / heads
+    input channels per head; rows q | k | v) and b_heads, in place of w_qkv / b_qkv.  Weights ~ N(0, w_std^2 * heads)
+    (a head sees 1/heads of the channels)."""
+    out = make_inputs(cfg, layer=layer, batch=batch, tensors=("x", "w_proj", "b_proj", "bias_table", "dy"))
+    nh, ds = cfg.num_heads, cfg.head_dim
+    dq = cfg.qk_dim or ds
+    out["w_heads"] = _normal(cfg.seed, layer, "w_heads", (nh, 2 * dq + ds, ds), cfg.w_std * float(nh) ** 0.5)
+    out["b_heads"] = _normal(cfg.seed, layer, "b_heads", (nh, 2 * dq + ds), cfg.bias_std) if cfg.bias_std > 0 else np.zeros((nh, 2 * dq + ds), np.float32)
+    if cfg.dtype == "bf16":
+        out = {k: round_to_bf16(v) for k, v in out.items()}
     return out
 
 
