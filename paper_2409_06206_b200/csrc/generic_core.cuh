@@ -325,5 +325,37 @@ inline HeadShifts head_shifts(const Plan& p) {
   return hs;
 }
 
+// ------------------------------------------------------------------------------------------
+// small element-wise helpers
+// ------------------------------------------------------------------------------------------
+// out[row, 0..w) = a[row*lda + 0..w) + b[row*ldb + 0..w)   (b may be null)
+template <typename T>
+__global__ void __launch_bounds__(256) add_cols_kernel(const T* __restrict__ a, long long lda, const T* __restrict__ b, long long ldb,
+                                                       T* __restrict__ out, long long ldo, long long rows, int w) {
+  const long long n = rows * w;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / w;
+    const int c = (int)(i - r * w);
+    float v = ldf(a + r * lda + c);
+    if (b != nullptr) v += ldf(b + r * ldb + c);
+    stf(out + r * ldo + c, v);
+  }
+}
+
+inline int grid_for(long long work_items, int per_block) {
+  long long g = (work_items + per_block - 1) / per_block;
+  const long long cap = (long long)device_sm_count() * 8;
+  if (g > cap) g = cap;
+  return g < 1 ? 1 : (int)g;
+}
+
+template <typename T>
+int launch_add_cols(const T* a, long long lda, const T* b, long long ldb, T* out, long long ldo, long long rows, int w,
+                    cudaStream_t st) {
+  { KernelScope ks_("add_cols", st);
+    add_cols_kernel<T><<<grid_for(rows * w, 256 * 8), 256, 0, st>>>(a, lda, b, ldb, out, ldo, rows, w); }
+  return check_launch();
+}
+
 }  // namespace generic
 }  // namespace gswa
